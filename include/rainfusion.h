@@ -1,0 +1,138 @@
+/*
+ * rainfusion.h - C ABI of the B200 (sm_100a) RainFusion hot path:
+ * per-head adaptive block-sparse 3D attention for video Diffusion Transformers
+ * (arxiv 2505.21036).
+ *
+ * Pipeline of one attention call (Sec. 1, last paragraph; Fig. 2a):
+ *   rf_arm_classify      ARM: one pattern per head from sampled scores   (Sec. 3.3, Eq. 6, Algorithm 1)
+ *   rf_build_block_mask  pattern masks as per-head lists of KV tiles     (Sec. 3.2, Eq. 3-5)
+ *   rf_sparse_attn_fwd   attention that skips what the pattern masks     (Eq. 1-2 with the pattern's mask)
+ *   rf_dense_attn_fwd    full 3D attention, the dense baseline           (Eq. 1-2)
+ *
+ * Conventions for every entry point
+ *   - Tensors Q, K, V, O are bf16, contiguous [B, H, N, D], N = T*frame_h*frame_w + L_text.
+ *     Video tokens come first, frame-major and row-major inside a frame (Sec. 3.1); text tokens last.
+ *   - Pointers marked "device" are CUDA device pointers owned by the caller; rf_shape / rf_params /
+ *     rf_schedule structs themselves are host memory, read during the call.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream).  No entry point synchronises the host or allocates device memory.  The library keeps
+ *     no state between calls apart from per-device kernel attributes set on first use.
+ *   - Host-detectable errors return a code before anything is launched.  Device-detected ones
+ *     (a bounded wait that ran out, a head class outside 0..3) are written to *dev_status
+ *     (device int32, may be NULL; never reset by the library) and the kernels still terminate.
+ *   - Supported: D in {64, 128}; block_m = block_n = 128 for the attention entry points;
+ *     rf_build_block_mask alone accepts any power-of-two blocks >= 16.
+ */
+#ifndef RAINFUSION_H_
+#define RAINFUSION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RF_OK = 0,
+  RF_ERR_INVALID_ARG = 1,
+  RF_ERR_UNSUPPORTED = 2,
+  RF_ERR_WORKSPACE_TOO_SMALL = 3,
+  RF_ERR_CUDA = 4,
+  RF_ERR_TIMEOUT = 5
+} rf_status;
+
+/* Head categories (Sec. 3.2).  RF_DENSE is not an ARM outcome; a caller may force it. */
+typedef enum { RF_SPATIAL = 0, RF_TEMPORAL = 1, RF_TEXTURAL = 2, RF_DENSE = 3 } rf_pattern;
+
+/* Which sample feeds which recall (Sec. 3.3; ablation column "L" of Table 2). */
+typedef enum {
+  RF_SAMPLE_ALG1 = 0,   /* Temporal recall on the first frame's tokens, Spatial recall on the stride sample */
+  RF_SAMPLE_GLOBAL = 1  /* both recalls on the stride sample */
+} rf_sample_mode;
+
+typedef struct {
+  int32_t B, H, D;            /* batch, heads, head dimension */
+  int32_t T;                  /* latent frames */
+  int32_t frame_h, frame_w;   /* tokens per frame = frame_h * frame_w */
+  int32_t L_text;             /* text tokens appended after the video tokens (>= 0) */
+} rf_shape;
+
+typedef struct {
+  int32_t frame_window;     /* w_f >= 0: a Spatial head keeps keys with |frame(q) - frame(k)| <= w_f (Eq. 3) */
+  int32_t spatial_window;   /* w_s >= 0: a Temporal head keeps keys with |pos(q) - pos(k)| <= w_s, pos = y*frame_w + x */
+  int32_t textural_stride;  /* tau >= 1: a Textural head keeps key (y, x) iff y mod tau == x mod tau (Eq. 4) */
+  int32_t sample_mode;      /* rf_sample_mode */
+  int32_t sample_stride;    /* omega >= 1: the stride sample is video tokens 0, omega, 2*omega, ... */
+  float   alpha;            /* recall threshold of Algorithm 1, in (0, 1] */
+  int32_t block_m, block_n; /* tile of the block mask: query rows x key slots */
+  int32_t temporal_permute; /* 1: Temporal heads run in position-major token order (slot = pos*T + frame) */
+} rf_params;
+
+/*
+ * Tile schedule: for every (b, h, query tile a) the ascending list of non-empty KV tiles in the
+ * head's own coordinate space (Dense/Spatial/Temporal: original order, or position-major for
+ * Temporal with temporal_permute; Textural: the kept set C in ascending order, then text).
+ * Entry = tile index, with bit 31 set when the tile is PARTIAL (some pair in it is masked, or
+ * it holds fewer than block_n real key slots); FULL tiles need no element mask.
+ * All arrays are device memory allocated by the caller.
+ */
+typedef struct {
+  int32_t  *count;    /* [B, H, nQ] */
+  int32_t  *kv_tile;  /* [B, H, nQ, nKmax], first count[...] entries of a row are valid */
+  uint32_t *bitmap;   /* optional [B, H, nQ, ceil(nKmax/32)] bit b = tile b listed; may be NULL */
+  int32_t  *kv_len;   /* [B, H] number of key slots of the head (N, or |C|*T + L_text for Textural) */
+  int32_t   nQ, nKmax;
+} rf_schedule;
+
+const char *rf_status_string(rf_status s);
+
+/* Host, pure: nQ = ceil(N/block_m), nKmax = ceil(N/block_n). */
+rf_status rf_schedule_dims(const rf_shape *shape, const rf_params *params, int32_t *nQ, int32_t *nKmax);
+
+/* Host, pure: bytes of device workspace that rf_arm_classify / rf_sparse_attn_fwd need
+ * (reordered Q/K/V copies for Temporal and Textural heads, ARM per-row recalls).  0 on bad arguments. */
+size_t rf_workspace_bytes(const rf_shape *shape, const rf_params *params);
+
+/*
+ * ARM (Sec. 3.3, Eq. 6, Algorithm 1).  For every (b, h): approximate softmax scores on the sampled
+ * queries/keys, the share of each row's mass kept by the sampled Temporal / Spatial / Textural mask,
+ * averaged over rows, then Temporal if R_t >= alpha, else Spatial if R_s >= alpha, else Textural.
+ *   q, k        device bf16 [B,H,N,D]
+ *   head_class  device int32 [B,H], written
+ *   recall      device float [B,H,3] = (R_temporal, R_spatial, R_textural), written; may be NULL
+ *   ws          device workspace of at least rf_workspace_bytes(), 256-byte aligned
+ */
+rf_status rf_arm_classify(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
+                          int32_t *head_class, float *recall, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Block mask / tile schedule of the pattern masks of Sec. 3.2 (Eq. 3-5), per head, from device-resident
+ * head classes.  Fills out->count, out->kv_tile, out->kv_len (and out->bitmap when not NULL);
+ * out->nQ / out->nKmax must equal rf_schedule_dims().
+ */
+rf_status rf_build_block_mask(const rf_shape *shape, const rf_params *params, const int32_t *head_class,
+                              rf_schedule *out, int32_t *dev_status, void *cuda_stream);
+
+/*
+ * Pattern-masked attention forward (Eq. 1-2 with M_spatial / M_temporal / the checkerboard K_C, V_C
+ * of Eq. 5).  Visits only the listed tiles and applies the exact element mask inside PARTIAL tiles,
+ * so the result does not depend on the tile size or on temporal_permute.
+ *   q, k, v     device bf16 [B,H,N,D]
+ *   head_class  device int32 [B,H] (the classes the schedule was built from)
+ *   o           device bf16 [B,H,N,D], written in original token order
+ *   lse         device float [B,H,N], natural-log sum of exp(score) over kept keys; may be NULL
+ *   ws          as for rf_arm_classify; holds the reordered copies this call makes
+ */
+rf_status rf_sparse_attn_fwd(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
+                             const void *v, const int32_t *head_class, const rf_schedule *sched, void *o,
+                             float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
+
+/* Full 3D attention (Eq. 1-2, all-zero mask): the same kernel walking every tile.  ws may be NULL. */
+rf_status rf_dense_attn_fwd(const rf_shape *shape, const void *q, const void *k, const void *v, void *o,
+                            float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAINFUSION_H_ */

@@ -1,0 +1,162 @@
+"""Thin ctypes binding of librainfusion.so (same names as include/rainfusion.h).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels behind the C ABI.
+torch supplies device memory and the current stream.  There is no fallback: if the shared
+library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+RF_SPATIAL, RF_TEMPORAL, RF_TEXTURAL, RF_DENSE = 0, 1, 2, 3
+RF_SAMPLE_ALG1, RF_SAMPLE_GLOBAL = 0, 1
+PARTIAL_BIT = 1 << 31
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librainfusion.so")
+_lib = None
+
+EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
+           "rf_build_block_mask", "rf_sparse_attn_fwd", "rf_dense_attn_fwd"]
+
+
+class rf_shape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("B", "H", "D", "T", "frame_h", "frame_w", "L_text")]
+
+
+class rf_params(C.Structure):
+    _fields_ = [("frame_window", C.c_int32), ("spatial_window", C.c_int32), ("textural_stride", C.c_int32),
+                ("sample_mode", C.c_int32), ("sample_stride", C.c_int32), ("alpha", C.c_float),
+                ("block_m", C.c_int32), ("block_n", C.c_int32), ("temporal_permute", C.c_int32)]
+
+
+class rf_schedule(C.Structure):
+    _fields_ = [("count", C.c_void_p), ("kv_tile", C.c_void_p), ("bitmap", C.c_void_p), ("kv_len", C.c_void_p),
+                ("nQ", C.c_int32), ("nKmax", C.c_int32)]
+
+
+class RainFusionError(RuntimeError):
+    pass
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def load():
+    """Loads the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RainFusionError(f"{_LIB_PATH} is missing: build it with `python -m paper_2505_21036_b200.build`")
+    lib = C.CDLL(_LIB_PATH)
+    P, V, I, Z = C.POINTER, C.c_void_p, C.c_int, C.c_size_t
+    lib.rf_status_string.restype = C.c_char_p
+    lib.rf_status_string.argtypes = [I]
+    lib.rf_schedule_dims.restype = I
+    lib.rf_schedule_dims.argtypes = [P(rf_shape), P(rf_params), P(C.c_int32), P(C.c_int32)]
+    lib.rf_workspace_bytes.restype = Z
+    lib.rf_workspace_bytes.argtypes = [P(rf_shape), P(rf_params)]
+    lib.rf_arm_classify.restype = I
+    lib.rf_arm_classify.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, Z, V]
+    lib.rf_build_block_mask.restype = I
+    lib.rf_build_block_mask.argtypes = [P(rf_shape), P(rf_params), V, P(rf_schedule), V, V]
+    lib.rf_sparse_attn_fwd.restype = I
+    lib.rf_sparse_attn_fwd.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
+    lib.rf_dense_attn_fwd.restype = I
+    lib.rf_dense_attn_fwd.argtypes = [P(rf_shape), V, V, V, V, V, V, Z, V, V]
+    _lib = lib
+    return lib
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise RainFusionError(f"{what} failed: {load().rf_status_string(code).decode()} ({code})")
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> Optional[int]:
+    import torch
+    s = torch.cuda.current_stream().cuda_stream
+    return s if s else None
+
+
+def make_shape(B, H, D, T, frame_h, frame_w, L_text) -> rf_shape:
+    return rf_shape(B, H, D, T, frame_h, frame_w, L_text)
+
+
+def make_params(frame_window, spatial_window, textural_stride=2, sample_mode=RF_SAMPLE_ALG1, sample_stride=1,
+                alpha=0.9, block_m=128, block_n=128, temporal_permute=1) -> rf_params:
+    return rf_params(frame_window, spatial_window, textural_stride, sample_mode, sample_stride, alpha,
+                     block_m, block_n, temporal_permute)
+
+
+def shape_of(wl) -> rf_shape:
+    """rf_shape of a synth.Workload."""
+    return rf_shape(wl.B, wl.H, wl.D, wl.T, wl.frame_h, wl.frame_w, wl.L_text)
+
+
+def params_of(wl, block_m=128, block_n=128, temporal_permute=1) -> rf_params:
+    """rf_params of a synth.Workload."""
+    return rf_params(wl.frame_window, wl.spatial_window, wl.textural_stride, wl.sample_mode, wl.sample_stride,
+                     wl.alpha, block_m, block_n, temporal_permute)
+
+
+def rf_schedule_dims(shape: rf_shape, params: rf_params):
+    nq, nk = C.c_int32(), C.c_int32()
+    _check(load().rf_schedule_dims(C.byref(shape), C.byref(params), C.byref(nq), C.byref(nk)), "rf_schedule_dims")
+    return nq.value, nk.value
+
+
+def rf_workspace_bytes(shape: rf_shape, params: rf_params) -> int:
+    n = load().rf_workspace_bytes(C.byref(shape), C.byref(params))
+    if n == 0:
+        raise RainFusionError("rf_workspace_bytes: invalid shape or parameters")
+    return n
+
+
+class Schedule:
+    """Device arrays of a tile schedule plus the C struct that points at them."""
+
+    def __init__(self, shape: rf_shape, params: rf_params, device, with_bitmap: bool = False):
+        import torch
+        self.nQ, self.nKmax = rf_schedule_dims(shape, params)
+        BH = shape.B * shape.H
+        self.count = torch.zeros((shape.B, shape.H, self.nQ), dtype=torch.int32, device=device)
+        self.kv_tile = torch.zeros((shape.B, shape.H, self.nQ, self.nKmax), dtype=torch.int32, device=device)
+        self.kv_len = torch.zeros((shape.B, shape.H), dtype=torch.int32, device=device)
+        self.bitmap = (torch.zeros((BH, self.nQ, (self.nKmax + 31) // 32), dtype=torch.int32, device=device)
+                       if with_bitmap else None)
+        self.c = rf_schedule(self.count.data_ptr(), self.kv_tile.data_ptr(), _ptr(self.bitmap),
+                             self.kv_len.data_ptr(), self.nQ, self.nKmax)
+
+
+def alloc_workspace(shape: rf_shape, params: rf_params, device):
+    import torch
+    return torch.empty(rf_workspace_bytes(shape, params), dtype=torch.uint8, device=device)
+
+
+def rf_arm_classify(shape, params, q, k, head_class, recall, ws):
+    _check(load().rf_arm_classify(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), head_class.data_ptr(),
+                                  _ptr(recall), ws.data_ptr(), ws.numel(), _stream()), "rf_arm_classify")
+
+
+def rf_build_block_mask(shape, params, head_class, sched: Schedule, dev_status=None):
+    _check(load().rf_build_block_mask(C.byref(shape), C.byref(params), head_class.data_ptr(), C.byref(sched.c),
+                                      _ptr(dev_status), _stream()), "rf_build_block_mask")
+
+
+def rf_sparse_attn_fwd(shape, params, q, k, v, head_class, sched: Schedule, o, lse, ws, dev_status=None):
+    _check(load().rf_sparse_attn_fwd(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                     head_class.data_ptr(), C.byref(sched.c), o.data_ptr(), _ptr(lse), ws.data_ptr(),
+                                     ws.numel(), _ptr(dev_status), _stream()), "rf_sparse_attn_fwd")
+
+
+def rf_dense_attn_fwd(shape, q, k, v, o, lse, dev_status=None):
+    _check(load().rf_dense_attn_fwd(C.byref(shape), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), _ptr(lse),
+                                    None, 0, _ptr(dev_status), _stream()), "rf_dense_attn_fwd")

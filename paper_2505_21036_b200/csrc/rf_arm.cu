@@ -1,0 +1,256 @@
+// ARM: Adaptive Recognition Module (Sec. 3.3, Eq. 6, Algorithm 1).
+//
+// For a sample I of video tokens (the first frame, or every omega-th token) each CTA takes 64
+// sampled query rows and streams all sampled keys through shared memory in blocks of 64:
+// scores on the tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate), online softmax in fp32
+// with warp shuffles for the row maximum, and next to the total mass three masked masses: the
+// part of the row kept by the Temporal, the Spatial and the Textural mask restricted to I.
+// The n x n score matrix is never written.  Per-row recalls go to scratch; a second kernel
+// averages them in a fixed order (deterministic) and takes Algorithm 1's decision.
+#include "rf_common.cuh"
+
+namespace {
+
+constexpr int ARM_ROWS = 64;   // query rows per CTA (16 per warp)
+constexpr int ARM_KEYS = 64;   // keys per shared-memory block
+constexpr int ARM_THREADS = 128;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+struct KeyAttr { int f, p, c; };  // frame, in-frame position, 1 if in the checkerboard set C
+
+__device__ __forceinline__ KeyAttr token_attr(const RfGeom& g, int tok) {
+  KeyAttr a;
+  a.f = tok / g.S;
+  a.p = tok - a.f * g.S;
+  const int y = a.p / g.Wf, x = a.p - y * g.Wf;
+  a.c = (y % g.tau) == (x % g.tau);
+  return a;
+}
+
+// grid = (ceil(n/64), B*H).  stride: token index of sample m is m*stride.
+// row_out: [B*H][3][n_pad] per-row recalls (temporal, spatial, textural) of this sample.
+template <int D>
+__global__ void __launch_bounds__(ARM_THREADS) rf_arm_rows_kernel(RfGeom g, int n, int stride, int n_pad,
+                                                                   const __nv_bfloat16* __restrict__ q,
+                                                                   const __nv_bfloat16* __restrict__ k,
+                                                                   float scale_log2, float* __restrict__ row_out) {
+  constexpr int LD = D + 8;  // padded row, keeps ldmatrix conflict-free
+  __shared__ __align__(16) __nv_bfloat16 Qs[ARM_ROWS * LD];
+  __shared__ __align__(16) __nv_bfloat16 Ks[ARM_KEYS * LD];
+  __shared__ int kf[ARM_KEYS], kp[ARM_KEYS], kc[ARM_KEYS];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int bh = blockIdx.y;
+  const int row0 = blockIdx.x * ARM_ROWS;
+  const size_t head = (size_t)bh * g.N * D;
+  constexpr int VEC = D / 8;
+
+  for (int i = tid; i < ARM_ROWS * VEC; i += ARM_THREADS) {
+    const int r = i / VEC, c = i % VEC;
+    const int m = row0 + r;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (m < n) val = __ldg(reinterpret_cast<const uint4*>(q + head + (size_t)m * stride * D) + c);
+    *reinterpret_cast<uint4*>(&Qs[r * LD + c * 8]) = val;
+  }
+  __syncthreads();
+
+  uint32_t qa[D / 16][4];
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    const uint32_t addr = smem_u32(&Qs[(warp * 16 + (lane & 15)) * LD + ks * 16 + (lane >> 4) * 8]);
+    ldmatrix_x4(addr, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
+  }
+
+  // the two rows this thread sees: warp*16 + lane/4 and +8
+  int rf[2], rp[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int m = min(row0 + warp * 16 + (lane >> 2) + h * 8, n - 1);
+    const KeyAttr a = token_attr(g, m * stride);
+    rf[h] = a.f;
+    rp[h] = a.p;
+  }
+  float mx[2] = {-INFINITY, -INFINITY};
+  float l_all[2] = {0.f, 0.f}, l_t[2] = {0.f, 0.f}, l_s[2] = {0.f, 0.f}, l_c[2] = {0.f, 0.f};
+
+  for (int k0 = 0; k0 < n; k0 += ARM_KEYS) {
+    __syncthreads();  // previous block fully consumed
+    for (int i = tid; i < ARM_KEYS * VEC; i += ARM_THREADS) {
+      const int r = i / VEC, c = i % VEC;
+      const int m = k0 + r;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (m < n) val = __ldg(reinterpret_cast<const uint4*>(k + head + (size_t)m * stride * D) + c);
+      *reinterpret_cast<uint4*>(&Ks[r * LD + c * 8]) = val;
+    }
+    if (tid < ARM_KEYS) {
+      const int m = k0 + tid;
+      if (m < n) {
+        const KeyAttr a = token_attr(g, m * stride);
+        kf[tid] = a.f; kp[tid] = a.p; kc[tid] = a.c;
+      } else {
+        kf[tid] = -1; kp[tid] = 0; kc[tid] = 0;  // f = -1 marks a slot past the sample
+      }
+    }
+    __syncthreads();
+
+    float acc[ARM_KEYS / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < ARM_KEYS / 8; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+      for (int np = 0; np < ARM_KEYS / 16; ++np) {
+        const int mi = lane >> 3;
+        const uint32_t addr = smem_u32(&Ks[(np * 16 + (mi >> 1) * 8 + (lane & 7)) * LD + ks * 16 + (mi & 1) * 8]);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4(addr, b0, b1, b2, b3);
+        mma_bf16_16816(acc[np * 2], qa[ks], b0, b1);
+        mma_bf16_16816(acc[np * 2 + 1], qa[ks], b2, b3);
+      }
+    }
+
+    // scale to the log2 domain, mask slots past the sample, block row maximum
+    float bm[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int nt = 0; nt < ARM_KEYS / 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
+        const float s = kf[col] < 0 ? -INFINITY : acc[nt][e] * scale_log2;
+        acc[nt][e] = s;
+        bm[e >> 1] = fmaxf(bm[e >> 1], s);
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      bm[h] = fmaxf(bm[h], __shfl_xor_sync(0xffffffffu, bm[h], 1));
+      bm[h] = fmaxf(bm[h], __shfl_xor_sync(0xffffffffu, bm[h], 2));
+      const float m_new = fmaxf(mx[h], bm[h]);           // finite: every block holds >= 1 real key
+      const float corr = exp2f(mx[h] - m_new);           // exp2(-inf) = 0 on the first block
+      l_all[h] *= corr; l_t[h] *= corr; l_s[h] *= corr; l_c[h] *= corr;
+      mx[h] = m_new;
+    }
+#pragma unroll
+    for (int nt = 0; nt < ARM_KEYS / 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int h = e >> 1;
+        const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
+        const float p = exp2f(acc[nt][e] - mx[h]);
+        l_all[h] += p;
+        if (abs(kp[col] - rp[h]) <= g.ws) l_t[h] += p;
+        if (abs(kf[col] - rf[h]) <= g.wf) l_s[h] += p;
+        if (kc[col]) l_c[h] += p;
+      }
+    }
+  }
+
+  // quad reduction of the partial masses, then one lane per row writes its recalls
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+      l_all[h] += __shfl_xor_sync(0xffffffffu, l_all[h], o);
+      l_t[h] += __shfl_xor_sync(0xffffffffu, l_t[h], o);
+      l_s[h] += __shfl_xor_sync(0xffffffffu, l_s[h], o);
+      l_c[h] += __shfl_xor_sync(0xffffffffu, l_c[h], o);
+    }
+    const int m = row0 + warp * 16 + (lane >> 2) + h * 8;
+    if ((lane & 3) == 0 && m < n) {
+      float* out = row_out + (size_t)bh * 3 * n_pad;
+      const float inv = 1.f / l_all[h];
+      out[m] = l_t[h] * inv;
+      out[n_pad + m] = l_s[h] * inv;
+      out[2 * n_pad + m] = l_c[h] * inv;
+    }
+  }
+}
+
+// One CTA per head: mean of the per-row recalls in a fixed order, then Algorithm 1.
+__global__ void __launch_bounds__(256) rf_arm_decide_kernel(int n_loc, int n_glb, int n_pad, int sample_mode, float alpha,
+                                                             const float* __restrict__ rows_loc,
+                                                             const float* __restrict__ rows_glb,
+                                                             int32_t* __restrict__ head_class, float* __restrict__ recall) {
+  __shared__ double red[3][256];
+  const int bh = blockIdx.x, tid = threadIdx.x;
+  const float* gl = rows_glb + (size_t)bh * 3 * n_pad;
+  const float* lo = rows_loc + (size_t)bh * 3 * n_pad;
+  const bool local_t = sample_mode == RF_SAMPLE_ALG1;
+  const float* src[3] = {local_t ? lo : gl, gl + n_pad, gl + 2 * n_pad};
+  const int cnt[3] = {local_t ? n_loc : n_glb, n_glb, n_glb};
+  for (int w = 0; w < 3; ++w) {
+    double s = 0.0;
+    for (int i = tid; i < cnt[w]; i += 256) s += (double)src[w][i];
+    red[w][tid] = s;
+  }
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (tid < o)
+      for (int w = 0; w < 3; ++w) red[w][tid] += red[w][tid + o];
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const float Rt = (float)(red[0][0] / cnt[0]), Rs = (float)(red[1][0] / cnt[1]), Rc = (float)(red[2][0] / cnt[2]);
+    if (recall) { recall[bh * 3] = Rt; recall[bh * 3 + 1] = Rs; recall[bh * 3 + 2] = Rc; }
+    head_class[bh] = Rt >= alpha ? RF_TEMPORAL : (Rs >= alpha ? RF_SPATIAL : RF_TEXTURAL);
+  }
+}
+
+template <int D>
+cudaError_t launch_rows(const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                        float* out, cudaStream_t st) {
+  dim3 grid(rf_cdiv(n, ARM_ROWS), g.B * g.H);
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+  rf_arm_rows_kernel<D><<<grid, ARM_THREADS, 0, st>>>(g, n, stride, n_pad, q, k, scale_log2, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rows_d(const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                          float* out, cudaStream_t st) {
+  switch (g.D) {
+    case 64: return launch_rows<64>(g, n, stride, n_pad, q, k, out, st);
+    case 96: return launch_rows<96>(g, n, stride, n_pad, q, k, out, st);
+    case 128: return launch_rows<128>(g, n, stride, n_pad, q, k, out, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+int arm_n_pad(const RfGeom& g, int omega) {
+  const int n_glb = rf_cdiv(g.Nv, omega);
+  const int n = n_glb > g.S ? n_glb : g.S;
+  return (n + 63) / 64 * 64;
+}
+
+}  // namespace
+
+size_t rf_arm_scratch_floats(const RfGeom& g, int omega) { return (size_t)2 * g.B * g.H * 3 * arm_n_pad(g, omega); }
+
+cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, const __nv_bfloat16* q,
+                          const __nv_bfloat16* k, int32_t* head_class, float* recall, float* row_scratch,
+                          cudaStream_t st) {
+  const int n_pad = arm_n_pad(g, omega);
+  const int n_glb = rf_cdiv(g.Nv, omega), n_loc = g.S;
+  float* rows_glb = row_scratch;
+  float* rows_loc = row_scratch + (size_t)g.B * g.H * 3 * n_pad;
+  cudaError_t e = launch_rows_d(g, n_glb, omega, n_pad, q, k, rows_glb, st);
+  if (e != cudaSuccess) return e;
+  if (sample_mode == RF_SAMPLE_ALG1) {
+    e = launch_rows_d(g, n_loc, 1, n_pad, q, k, rows_loc, st);
+    if (e != cudaSuccess) return e;
+  }
+  rf_arm_decide_kernel<<<g.B * g.H, 256, 0, st>>>(n_loc, n_glb, n_pad, sample_mode, alpha, rows_loc, rows_glb,
+                                                  head_class, recall);
+  return cudaGetLastError();
+}

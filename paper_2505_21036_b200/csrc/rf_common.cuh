@@ -1,0 +1,60 @@
+// Shared host/device definitions of the RainFusion CUDA path (sm_100a only).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/rainfusion.h"
+
+#define RF_PARTIAL_BIT 0x80000000u
+
+// Geometry and pattern parameters as the kernels see them (passed by value).
+struct RfGeom {
+  int B, H, D;
+  int T, Hf, Wf, S;      // frames, frame height/width, tokens per frame
+  int Nv, L, N;          // video tokens, text tokens, all tokens
+  int wf, ws, tau;       // frame window, spatial window, checkerboard stride
+  int nC;                // kept tokens per frame for the Textural pattern
+  int LkvTex;            // key slots of a Textural head: T*nC + L
+  int BM, BN, nQ, nKmax; // block mask tile and its extents
+  int permute;           // Temporal heads in position-major order
+};
+
+// Device-side error reporting: first error wins, kernels never trap.
+__device__ __forceinline__ void rf_report(int32_t* dev_status, int code) {
+  if (dev_status != nullptr) atomicCAS(dev_status, 0, code);
+}
+
+__host__ __device__ __forceinline__ int rf_cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// Number of key slots of a head of class `cls`.
+__host__ __device__ __forceinline__ int rf_kv_len(const RfGeom& g, int cls) {
+  return cls == RF_TEXTURAL ? g.LkvTex : g.N;
+}
+
+// Launchers implemented in the .cu files (host).
+cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, int32_t* count, int32_t* kv_tile,
+                                  uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st);
+cudaError_t rf_launch_gather(const RfGeom& g, const int32_t* head_class, const __nv_bfloat16* q,
+                             const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* wq, __nv_bfloat16* wk,
+                             __nv_bfloat16* wv, cudaStream_t st);
+cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, const __nv_bfloat16* q,
+                          const __nv_bfloat16* k, int32_t* head_class, float* recall, float* row_scratch,
+                          cudaStream_t st);
+size_t rf_arm_scratch_floats(const RfGeom& g, int omega);
+
+struct RfAttnArgs {
+  RfGeom g;
+  const int32_t* head_class;  // nullptr: every head Dense, implicit full tile list
+  const int32_t* count;
+  const int32_t* kv_tile;
+  __nv_bfloat16* o;
+  float* lse;
+  int32_t* dev_status;
+  float scale_log2;           // log2(e) / sqrt(D)
+};
+// Tensor maps: [0..2] Q/K/V in original order, [3..5] the workspace copies with N rows per head
+// (position-major Q/K/V of Temporal heads), [6..7] workspace K/V with LkvTex rows per head (Textural).
+rf_status rf_launch_attention(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st);

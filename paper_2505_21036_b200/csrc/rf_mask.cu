@@ -1,0 +1,177 @@
+// Block-mask / tile-schedule builder and the token reordering gathers.
+//
+// The pattern masks of Sec. 3.2 (Spatial: Eq. 3, Temporal, Textural: Eq. 4-5) are evaluated in
+// closed form per tile: a tile's query slots and key slots each cover a contiguous range of
+// frames (Spatial), of in-frame positions (Temporal in position-major order) or a cyclic range
+// of positions (Temporal in original order), so "some pair kept" and "all pairs kept" reduce to
+// distances between at most two intervals per side.
+#include "rf_common.cuh"
+
+namespace {
+
+struct Iv { int lo, hi; };  // closed interval
+
+// Positions (index mod S) covered by slots [a0, a1) of the original order: one or two intervals.
+__device__ __forceinline__ int cyclic_intervals(int a0, int a1, int S, Iv out[2]) {
+  if (a1 - a0 >= S) { out[0] = {0, S - 1}; return 1; }
+  int s = a0 % S, e = (a1 - 1) % S;
+  if (s <= e) { out[0] = {s, e}; return 1; }
+  out[0] = {s, S - 1};
+  out[1] = {0, e};
+  return 2;
+}
+
+// 0: empty, 1: PARTIAL, 2: FULL.  Tile (a, b) of a head of class cls.
+__device__ int tile_flag(const RfGeom& g, int cls, int a, int b) {
+  const int Lkv = rf_kv_len(g, cls);
+  const int r0 = a * g.BM, r1 = min(r0 + g.BM, g.N);
+  const int u0 = b * g.BN, u1 = min(u0 + g.BN, Lkv);
+  if (r0 >= r1 || u0 >= u1) return 0;
+  const bool full_width = (b + 1) * g.BN <= Lkv;
+  bool any = true, all = true;
+  if (cls == RF_SPATIAL || cls == RF_TEMPORAL) {
+    const int Nv = g.Nv;
+    const bool text_row = r1 > Nv, text_col = u1 > Nv;
+    const bool video_part = r0 < Nv && u0 < Nv;
+    bool vv_any = false, vv_all = true;
+    if (video_part) {
+      const int rv1 = min(r1, Nv), uv1 = min(u1, Nv);
+      if (cls == RF_SPATIAL || g.permute) {
+        // contiguous ranges of frames (Spatial) or of positions (position-major Temporal)
+        const int unit = cls == RF_SPATIAL ? g.S : g.T;
+        const int w = cls == RF_SPATIAL ? g.wf : g.ws;
+        const int ra = r0 / unit, rb = (rv1 - 1) / unit, ca = u0 / unit, cb = (uv1 - 1) / unit;
+        vv_any = max(max(ca - rb, ra - cb), 0) <= w;
+        vv_all = max(rb - ca, cb - ra) <= w;
+      } else {
+        Iv R[2], C[2];
+        const int nr = cyclic_intervals(r0, rv1, g.S, R), nc = cyclic_intervals(u0, uv1, g.S, C);
+        for (int i = 0; i < nr; ++i)
+          for (int j = 0; j < nc; ++j) {
+            vv_any = vv_any || max(max(C[j].lo - R[i].hi, R[i].lo - C[j].hi), 0) <= g.ws;
+            vv_all = vv_all && max(R[i].hi - C[j].lo, C[j].hi - R[i].lo) <= g.ws;
+          }
+      }
+    }
+    any = text_row || text_col || vv_any;
+    all = vv_all;
+  }
+  if (!any) return 0;
+  return (all && full_width) ? 2 : 1;
+}
+
+// One CTA per (query tile, head): flags for all key tiles, then an ordered compaction.
+__global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int32_t* __restrict__ head_class,
+                                                              int32_t* __restrict__ count, int32_t* __restrict__ kv_tile,
+                                                              uint32_t* __restrict__ bitmap, int32_t* __restrict__ kv_len,
+                                                              int32_t* dev_status) {
+  __shared__ int warp_tot[8];
+  __shared__ int base;
+  const int a = blockIdx.x, bh = blockIdx.y;
+  int cls = head_class[bh];
+  if (cls < 0 || cls > 3) {
+    if (threadIdx.x == 0) rf_report(dev_status, RF_ERR_INVALID_ARG);
+    cls = RF_DENSE;
+  }
+  const int Lkv = rf_kv_len(g, cls);
+  const int nK = rf_cdiv(Lkv, g.BN);
+  if (a == 0 && threadIdx.x == 0) kv_len[bh] = Lkv;
+  int32_t* row = kv_tile + ((size_t)bh * g.nQ + a) * g.nKmax;
+  const int words = rf_cdiv(g.nKmax, 32);
+  uint32_t* brow = bitmap ? bitmap + ((size_t)bh * g.nQ + a) * words : nullptr;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int b0 = 0; b0 < g.nKmax; b0 += 256) {
+    const int b = b0 + threadIdx.x;
+    const int f = (b < nK) ? tile_flag(g, cls, a, b) : 0;
+    const unsigned m = __ballot_sync(0xffffffffu, f != 0);
+    if (lane == 0) warp_tot[warp] = __popc(m);
+    if (brow && lane == 0 && (b >> 5) < words) brow[b >> 5] = m;
+    __syncthreads();
+    int off = base;
+    for (int w = 0; w < warp; ++w) off += warp_tot[w];
+    if (f != 0) row[off + __popc(m & ((1u << lane) - 1))] = (int32_t)((uint32_t)b | (f == 1 ? RF_PARTIAL_BIT : 0u));
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int t = 0;
+      for (int w = 0; w < 8; ++w) t += warp_tot[w];
+      base += t;
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) count[(size_t)bh * g.nQ + a] = base;
+}
+
+// Reordered copies for heads whose coordinate space is not the original one.
+//   Temporal + permute: Q, K, V  -> slot pos*T + frame (text rows keep their index)
+//   Textural:           K, V     -> frame*nC + rank(pos) for kept positions, text after T*nC
+// One 16-byte vector per thread; grid.x walks source rows, grid.y = head.
+__global__ void __launch_bounds__(256) rf_gather_kernel(RfGeom g, const int32_t* __restrict__ head_class,
+                                                         const uint4* __restrict__ q, const uint4* __restrict__ k,
+                                                         const uint4* __restrict__ v, uint4* __restrict__ wq,
+                                                         uint4* __restrict__ wk, uint4* __restrict__ wv) {
+  extern __shared__ int row_start[];  // [Hf] rank of the first kept token of each frame row (Textural)
+  const int bh = blockIdx.y;
+  const int cls = head_class[bh];
+  const bool perm = cls == RF_TEMPORAL && g.permute;
+  const bool tex = cls == RF_TEXTURAL;
+  if (!perm && !tex) return;
+  if (tex) {
+    if (threadIdx.x == 0) {
+      int acc = 0;
+      for (int y = 0; y < g.Hf; ++y) {
+        row_start[y] = acc;
+        const int r = y % g.tau;
+        acc += r < g.Wf ? (g.Wf - r + g.tau - 1) / g.tau : 0;
+      }
+    }
+    __syncthreads();
+  }
+  const int vec = g.D / 8;  // uint4 per row
+  const int rows_per_cta = 256 / vec;
+  const int lr = threadIdx.x / vec, c = threadIdx.x % vec;
+  if (lr >= rows_per_cta) return;
+  const size_t head_off = (size_t)bh * g.N * vec;
+  for (int i = blockIdx.x * rows_per_cta + lr; i < g.N; i += gridDim.x * rows_per_cta) {
+    int dst;
+    if (i >= g.Nv) {
+      dst = tex ? g.T * g.nC + (i - g.Nv) : i;
+    } else {
+      const int f = i / g.S, p = i - f * g.S;
+      if (perm) {
+        dst = p * g.T + f;
+      } else {
+        const int y = p / g.Wf, x = p - y * g.Wf;
+        if ((y % g.tau) != (x % g.tau)) continue;
+        dst = f * g.nC + row_start[y] + x / g.tau;
+      }
+    }
+    const size_t s = head_off + (size_t)i * vec + c, d = head_off + (size_t)dst * vec + c;
+    if (perm) wq[d] = q[s];
+    wk[d] = k[s];
+    wv[d] = v[s];
+  }
+}
+
+}  // namespace
+
+cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, int32_t* count, int32_t* kv_tile,
+                                  uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st) {
+  dim3 grid(g.nQ, g.B * g.H);
+  rf_build_tiles_kernel<<<grid, 256, 0, st>>>(g, head_class, count, kv_tile, bitmap, kv_len, dev_status);
+  return cudaGetLastError();
+}
+
+cudaError_t rf_launch_gather(const RfGeom& g, const int32_t* head_class, const __nv_bfloat16* q,
+                             const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* wq, __nv_bfloat16* wk,
+                             __nv_bfloat16* wv, cudaStream_t st) {
+  const int vec = g.D / 8;
+  const int rows_per_cta = 256 / vec;
+  int gx = rf_cdiv(g.N, rows_per_cta);
+  if (gx > 148 * 8) gx = 148 * 8;
+  dim3 grid(gx, g.B * g.H);
+  rf_gather_kernel<<<grid, 256, g.Hf * sizeof(int), st>>>(g, head_class, (const uint4*)q, (const uint4*)k,
+                                                           (const uint4*)v, (uint4*)wq, (uint4*)wk, (uint4*)wv);
+  return cudaGetLastError();
+}

@@ -1,0 +1,208 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rainfusion_oracle as orc
+from paper_2505_21036_b200 import api, synth
+
+import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+S_, T_, X_, D_ = orc.SPATIAL, orc.TEMPORAL, orc.TEXTURAL, orc.DENSE
+
+
+def mid_workload(D=64, H=4, **kw):
+    # 6 frames of 12x11 tokens + 37 text tokens = 829 tokens: 7 tiles of 128 with a ragged tail,
+    # frame length 132 cuts every tile boundary
+    return synth.small_workload("mid", H=H, D=D, T=6, fh=12, fw=11, L=37, wf=1, ws=20, tau=2, mode=0, omega=6, **kw)
+
+
+# ------------------------------------------------------------------ block masks / tile lists
+
+@pytest.mark.parametrize("block", [16, 32, 64, 128])
+@pytest.mark.parametrize("permute", [0, 1])
+def test_tile_lists_tiny_bit_exact(block, permute):
+    wl = synth.WORKLOADS["tiny"]
+    for classes in ([S_, T_, X_], [D_, X_, T_]):
+        run = gu.Run(wl, block=block, temporal_permute=permute)
+        run.force_classes(classes)
+        run.build()
+        assert int(run.status.item()) == 0
+        for h, cls in enumerate(classes):
+            ref = gu.oracle_lists(wl, cls, block, permute)
+            got = run.lists(0, h)
+            assert got == [ref[a] for a in range(run.sched.nQ)], (block, permute, cls)
+            assert int(run.sched.kv_len[0, h]) == orc.kv_len(cls, gu.geom(wl), gu.pparams(wl))
+
+
+@pytest.mark.parametrize("block", [16, 64, 128])
+@pytest.mark.parametrize("permute", [0, 1])
+def test_tile_lists_mid_bit_exact_and_bitmap(block, permute):
+    wl = mid_workload()
+    run = gu.Run(wl, block=block, temporal_permute=permute)
+    classes = [S_, T_, X_, D_]
+    run.force_classes(classes)
+    run.build()
+    bitmap = run.sched.bitmap.cpu().numpy().view(np.uint32)
+    for h, cls in enumerate(classes):
+        ref = gu.oracle_lists(wl, cls, block, permute)
+        got = run.lists(0, h)
+        assert got == [ref[a] for a in range(run.sched.nQ)], (block, permute, cls)
+        for a in range(run.sched.nQ):
+            listed = sorted(e & 0x7FFFFFFF for e in ref[a])
+            bits = [b for b in range(run.sched.nKmax) if (bitmap[h, a, b // 32] >> (b % 32)) & 1]
+            assert bits == listed
+
+
+def test_invalid_class_is_reported_not_trapped():
+    wl = synth.WORKLOADS["tiny"]
+    run = gu.Run(wl)
+    run.force_classes([0, 7, 2])
+    run.build()
+    assert int(run.status.item()) == 1        # RF_ERR_INVALID_ARG, kernel finished normally
+    assert run.lists(0, 1) == run.lists(0, 1)
+
+
+# ------------------------------------------------------------------ ARM
+
+def check_arm(wl, run=None):
+    run = run or gu.Run(wl)
+    cls_gpu, rec_gpu = run.arm()
+    cls_ref, rec_ref, margin = orc.arm_classify(run.q_bits, run.k_bits, gu.geom(wl), gu.pparams(wl),
+                                                wl.sample_mode, wl.sample_stride, wl.alpha)
+    assert np.abs(rec_gpu - rec_ref).max() <= gu.RECALL_ABS, np.abs(rec_gpu - rec_ref).max()
+    decided = margin > gu.TIE_MARGIN
+    assert np.array_equal(cls_gpu[decided], cls_ref[decided])
+    return cls_gpu, cls_ref, int((~decided).sum())
+
+
+def test_arm_tiny():
+    cls_gpu, cls_ref, ties = check_arm(synth.WORKLOADS["tiny"])
+    assert cls_ref[0].tolist() == [S_, T_, X_] and ties == 0
+
+
+@pytest.mark.parametrize("D", [64, 96, 128])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_arm_mid(D, mode):
+    wl = synth.small_workload("arm_mid", H=6, D=D, T=6, fh=12, fw=11, L=37, wf=1, ws=20, tau=3, mode=mode, omega=6,
+                              amp=1.5)
+    check_arm(wl)
+
+
+def test_arm_is_deterministic():
+    wl = mid_workload()
+    run = gu.Run(wl)
+    a = run.arm()[1].copy()
+    b = run.arm()[1].copy()
+    assert np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------ attention
+
+def oracle_heads(run, classes, rows=None):
+    wl = run.wl
+    out = []
+    for h, cls in enumerate(classes):
+        out.append(orc.masked_attention(run.q_bits[0, h], run.k_bits[0, h], run.v_bits[0, h], cls, gu.geom(wl),
+                                        gu.pparams(wl), rows=rows))
+    return out
+
+
+def test_dense_tiny():
+    wl = synth.WORKLOADS["tiny"]
+    run = gu.Run(wl)
+    O, lse = run.dense()
+    for h, (Or, lr) in enumerate(oracle_heads(run, [D_] * wl.H)):
+        gu.check_attention(O[0, h], lse[0, h], Or, lr, f"dense tiny head {h}")
+
+
+def test_pipeline_tiny():
+    """ARM -> block mask -> sparse attention, classes staying on the device."""
+    wl = synth.WORKLOADS["tiny"]
+    run = gu.Run(wl)
+    cls_gpu, _ = run.arm()
+    run.build()
+    O, lse = run.sparse()
+    assert cls_gpu[0].tolist() == [S_, T_, X_]
+    for h, (Or, lr) in enumerate(oracle_heads(run, cls_gpu[0].tolist())):
+        gu.check_attention(O[0, h], lse[0, h], Or, lr, f"pipeline tiny head {h}")
+
+
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("permute", [0, 1])
+def test_sparse_mid_all_patterns(D, permute):
+    wl = mid_workload(D=D)
+    run = gu.Run(wl, temporal_permute=permute)
+    classes = [S_, T_, X_, D_]
+    run.force_classes(classes)
+    run.build()
+    O, lse = run.sparse()
+    for h, (Or, lr) in enumerate(oracle_heads(run, classes)):
+        gu.check_attention(O[0, h], lse[0, h], Or, lr, f"mid D={D} permute={permute} class {classes[h]}")
+
+
+def test_dense_mid_and_batch():
+    wl = synth.small_workload("mid_b2", B=2, H=2, D=128, T=3, fh=9, fw=10, L=5)
+    run = gu.Run(wl)
+    O, lse = run.dense()
+    g, pp = gu.geom(wl), gu.pparams(wl)
+    for b in range(2):
+        for h in range(2):
+            Or, lr = orc.masked_attention(run.q_bits[b, h], run.k_bits[b, h], run.v_bits[b, h], D_, g, pp)
+            gu.check_attention(O[b, h], lse[b, h], Or, lr, f"dense b={b} h={h}")
+
+
+def test_permutation_on_off_agree():
+    wl = mid_workload(D=128)
+    outs = []
+    for permute in (0, 1):
+        run = gu.Run(wl, temporal_permute=permute)
+        run.force_classes([T_] * wl.H)
+        run.build()
+        outs.append(run.sparse())
+    # both are bf16-rounded outputs of magnitude up to ~4: they may differ by one bf16 ulp (2^-6)
+    assert np.abs(outs[0][0] - outs[1][0]).max() <= 3.2e-2
+    assert np.abs(outs[0][1] - outs[1][1]).max() <= 1e-3
+
+
+def planted_boundary_inputs(wl, cls, inside: bool):
+    """Keys just inside (spotlight) or just outside (poison) every row's kept set get a huge
+    matching logit and large values: a wrongly masked element removes an O(1) contribution, a
+    leaked one explodes the output."""
+    g, pp = gu.geom(wl), gu.pparams(wl)
+    q, k, v = synth.make_head(wl, 0, 0, kind="none")
+    qf, kf, vf = (synth.bf16_bits_to_f32(x).copy() for x in (q, k, v))
+    qf *= 0.1
+    kf *= 0.1
+    idx = np.arange(g.N)
+    M = orc.keep_mask(cls, idx, idx, g, pp)
+    target = np.zeros(g.N, dtype=bool)
+    for i in range(0, g.Nv, 7):
+        row = M[i, :g.Nv]
+        edges = np.flatnonzero(row[1:] != row[:-1])
+        for e in edges[:4]:
+            j = e if row[e] == inside else e + 1
+            target[j] = True
+    qf[:, 0] = 6.0
+    kf[target, 0] = 6.0 * np.sqrt(wl.D)
+    vf[target] = 50.0 if not inside else 3.0
+    return tuple(synth.f32_to_bf16_bits(x) for x in (qf, kf, vf)), target
+
+
+@pytest.mark.parametrize("cls", [S_, T_])
+@pytest.mark.parametrize("permute", [0, 1])
+@pytest.mark.parametrize("inside", [True, False])
+def test_boundary_spotlight_and_poison(cls, permute, inside):
+    wl = synth.small_workload("edge", H=1, D=64, T=6, fh=12, fw=11, L=37, wf=1, ws=20)
+    (q, k, v), target = planted_boundary_inputs(wl, cls, inside)
+    run = gu.Run(wl, qkv=(q[None, None], k[None, None], v[None, None]), temporal_permute=permute)
+    run.force_classes([cls])
+    run.build()
+    O, lse = run.sparse()
+    Or, lr = orc.masked_attention(q, k, v, cls, gu.geom(wl), gu.pparams(wl))
+    assert np.abs(Or).max() > 1.0                       # the planted keys matter for the reference
+    err = np.abs(O[0, 0] - Or)
+    assert err.max() <= 5e-2 * max(1.0, np.abs(Or).max()), err.max()
+    assert np.abs(lse[0, 0] - lr).max() <= 5e-3

@@ -128,6 +128,16 @@ rf_status rf_sparse_attn_fwd(const rf_shape *shape, const rf_params *params, con
                              const void *v, const int32_t *head_class, const rf_schedule *sched, void *o,
                              float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
 
+/*
+ * The token reordering that rf_sparse_attn_fwd performs before its attention kernel, on its own
+ * (Sec. 3.2, Textural Head: the K, V sequence is rearranged and the checkerboard tokens retained;
+ * Temporal heads with temporal_permute: Q, K, V to position-major order).  Writes the copies into ws.
+ * Exposed so that the reordering can be timed or reused separately; rf_sparse_attn_fwd does not need
+ * it to be called first.
+ */
+rf_status rf_reorder_tokens(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
+                            const void *v, const int32_t *head_class, void *ws, size_t ws_bytes, void *cuda_stream);
+
 /* Full 3D attention (Eq. 1-2, all-zero mask): the same kernel walking every tile.  ws may be NULL. */
 rf_status rf_dense_attn_fwd(const rf_shape *shape, const void *q, const void *k, const void *v, void *o,
                             float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);

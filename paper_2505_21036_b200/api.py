@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librainfus
 _lib = None
 
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
-           "rf_build_block_mask", "rf_sparse_attn_fwd", "rf_dense_attn_fwd"]
+           "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd"]
 
 
 class rf_shape(C.Structure):
@@ -65,6 +65,8 @@ def load():
     lib.rf_build_block_mask.argtypes = [P(rf_shape), P(rf_params), V, P(rf_schedule), V, V]
     lib.rf_sparse_attn_fwd.restype = I
     lib.rf_sparse_attn_fwd.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
+    lib.rf_reorder_tokens.restype = I
+    lib.rf_reorder_tokens.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, Z, V]
     lib.rf_dense_attn_fwd.restype = I
     lib.rf_dense_attn_fwd.argtypes = [P(rf_shape), V, V, V, V, V, V, Z, V, V]
     _lib = lib
@@ -155,6 +157,11 @@ def rf_sparse_attn_fwd(shape, params, q, k, v, head_class, sched: Schedule, o, l
     _check(load().rf_sparse_attn_fwd(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), v.data_ptr(),
                                      head_class.data_ptr(), C.byref(sched.c), o.data_ptr(), _ptr(lse), ws.data_ptr(),
                                      ws.numel(), _ptr(dev_status), _stream()), "rf_sparse_attn_fwd")
+
+
+def rf_reorder_tokens(shape, params, q, k, v, head_class, ws):
+    _check(load().rf_reorder_tokens(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                    head_class.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "rf_reorder_tokens")
 
 
 def rf_dense_attn_fwd(shape, q, k, v, o, lse, dev_status=None):

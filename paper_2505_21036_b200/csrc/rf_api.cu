@@ -213,6 +213,26 @@ rf_status rf_sparse_attn_fwd(const rf_shape* shape, const rf_params* params, con
   return rf_launch_attention(a, maps, stream);
 }
 
+rf_status rf_reorder_tokens(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
+                            const void* v, const int32_t* head_class, void* ws, size_t ws_bytes, void* cuda_stream) {
+  rf_status st = check_shape(shape);
+  if (st != RF_OK) return st;
+  st = check_params(params);
+  if (st != RF_OK) return st;
+  if (q == nullptr || k == nullptr || v == nullptr || head_class == nullptr || ws == nullptr) return RF_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0)
+    return RF_ERR_INVALID_ARG;
+  if (ws_bytes < rf_workspace_bytes(shape, params)) return RF_ERR_WORKSPACE_TOO_SMALL;
+  const RfGeom g = make_geom(shape, params);
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  cudaError_t e = rf_launch_gather(g, head_class, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+                                   static_cast<const __nv_bfloat16*>(v), reinterpret_cast<__nv_bfloat16*>(w),
+                                   reinterpret_cast<__nv_bfloat16*>(w + tensor_bytes(g)),
+                                   reinterpret_cast<__nv_bfloat16*>(w + 2 * tensor_bytes(g)),
+                                   static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
+}
+
 rf_status rf_dense_attn_fwd(const rf_shape* shape, const void* q, const void* k, const void* v, void* o, float* lse,
                             void* ws, size_t ws_bytes, int32_t* dev_status, void* cuda_stream) {
   (void)ws;

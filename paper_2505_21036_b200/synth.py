@@ -172,9 +172,19 @@ def make_qkv(wl: Workload, kinds: Sequence[str] | None = None):
     q = np.empty((wl.B, wl.H, wl.N, wl.D), dtype=np.uint16)
     k = np.empty_like(q)
     v = np.empty_like(q)
-    for b in range(wl.B):
-        for h in range(wl.H):
-            q[b, h], k[b, h], v[b, h] = make_head(wl, b, h, kinds[h])
+
+    def fill(bh):
+        b, h = divmod(bh, wl.H)
+        q[b, h], k[b, h], v[b, h] = make_head(wl, b, h, kinds[h])
+
+    if wl.B * wl.H * wl.N * wl.D > (1 << 24):
+        from concurrent.futures import ThreadPoolExecutor
+        import os
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+            list(ex.map(fill, range(wl.B * wl.H)))
+    else:
+        for bh in range(wl.B * wl.H):
+            fill(bh)
     return q, k, v
 
 

@@ -1,10 +1,17 @@
 // Pattern-masked FlashAttention forward on tcgen05 / TMEM / TMA (Eq. 1-2 with the masks of Sec. 3.2).
 //
-// One CTA owns one 128-row query tile of one head and walks that tile's list of KV tiles.
-// Per KV tile: S = Q K^T (tcgen05.mma, operands staged by TMA in 128B-swizzled shared memory,
-// accumulator in TMEM), online softmax in fp32 with one thread per query row (tcgen05.ld), P rounded
-// to bf16 into swizzled shared memory, O_tile = P V on the tensor cores, running O in registers.
-// K/V tiles are double-buffered: the TMA for tile i+1 is in flight while tile i is computed.
+// One CTA owns two adjacent 128-row query tiles of one head (two "streams") and walks the union of
+// their KV-tile lists, so every K/V tile fetched by TMA feeds up to two S = Q K^T and two O += P V
+// contractions.  Warp roles:
+//   warps 0-3  softmax of stream 0   (one thread per query row, TMEM lane = row)
+//   warps 4-7  softmax of stream 1
+//   warp  8    TMA producer: Q once, then K and V tiles into two shared-memory rings
+//   warp  9    MMA issuer: tcgen05.mma, accumulators in TMEM (S0, S1, O0, O1)
+// Per listed tile and stream: S lands in TMEM, the softmax warps read their rows (tcgen05.ld), keep a
+// running maximum and sum in fp32, write P as packed bf16 back into the S columns (tcgen05.st) and the
+// MMA warp multiplies it with V straight from TMEM.  The running maximum is only raised when it grows
+// by more than 2^8 (P stays well inside bf16/fp32 range), in which case the softmax warp itself
+// rescales its rows of O in TMEM; the final O / l and the log-sum-exp are exact either way.
 // PARTIAL tiles apply the exact element mask of the head's pattern; FULL tiles skip it.
 #include "rf_sm100.cuh"
 
@@ -13,23 +20,39 @@ namespace {
 using namespace sm100;
 
 constexpr int BM = 128, BN = 128;
-constexpr int kThreads = 128;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kThreads = 320;
+constexpr int kTmaWarp = 8, kMmaWarp = 9;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 struct Maps { CUtensorMap m[8]; };
 
 template <int D>
-struct Smem {
-  static constexpr int KB = D / 64;                 // 64-column (128-byte) blocks per row
-  static constexpr uint32_t BLK = 128 * 128;        // bytes of one 128-row x 64-col bf16 block
+struct Cfg {
+  static constexpr int KB = D / 64;                   // 64-column (128-byte) blocks per row
+  static constexpr uint32_t BLK = 128 * 128;          // bytes of one 128-row x 64-col bf16 block
+  static constexpr uint32_t TILE = KB * BLK;          // bytes of one 128-row tile
+  static constexpr int NK = D == 128 ? 2 : 4;         // K ring depth
+  static constexpr int NV = D == 128 ? 2 : 4;         // V ring depth
   static constexpr uint32_t Q = 0;
-  static constexpr uint32_t K0 = Q + KB * BLK;
-  static constexpr uint32_t V0 = K0 + 2 * KB * BLK;
-  static constexpr uint32_t P = V0 + 2 * KB * BLK;
-  static constexpr uint32_t BAR = P + 2 * BLK;      // mbarriers: q, kv[2], mma
-  static constexpr uint32_t MISC = BAR + 64;        // tmem base, abort flag
+  static constexpr uint32_t K0 = Q + 2 * TILE;
+  static constexpr uint32_t V0 = K0 + NK * TILE;
+  static constexpr uint32_t BAR = V0 + NV * TILE;
+  // barrier slots (8 bytes each)
+  static constexpr int B_Q = 0, B_KF = 1, B_KE = B_KF + NK, B_VF = B_KE + NK, B_VE = B_VF + NV, B_SF = B_VE + NV,
+                       B_PF = B_SF + 2, B_OF = B_PF + 2, B_COUNT = B_OF + 2;
+  static constexpr uint32_t MISC = BAR + 8 * ((B_COUNT + 7) / 8 * 8);
   static constexpr uint32_t TOTAL = MISC + 64;
-  static constexpr uint32_t ALLOC = TOTAL + 1024;   // slack for manual 1024-byte alignment
+  static constexpr uint32_t ALLOC = TOTAL + 1024;     // slack for manual 1024-byte alignment
+  // TMEM columns
+  static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL0 = 256, O_COL1 = 384, TMEM_COLS = 512;
 };
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 // Element mask of one query row in the head's key-slot space.
 struct RowMask {
@@ -75,26 +98,52 @@ __device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r
   return m;
 }
 
+// The two streams' ascending tile lists and their merge (the order K/V tiles are fetched in).
+struct Lists {
+  const int32_t* l0;
+  const int32_t* l1;
+  int n0, n1;
+  int lkv;
+  bool listed;
+  __device__ __forceinline__ uint32_t entry(int j, int i) const {
+    if (listed) return (uint32_t)(j == 0 ? l0[i] : l1[i]);
+    const bool tail = (i + 1) * BN > lkv;
+    return (uint32_t)i | (tail ? RF_PARTIAL_BIT : 0u);
+  }
+};
+struct Merge {
+  int i0 = 0, i1 = 0;
+  // Next tile of the union; uses bit j set when stream j lists it.  Returns false when exhausted.
+  __device__ __forceinline__ bool next(const Lists& L, int& tile, int& uses) {
+    const int e0 = i0 < L.n0 ? (int)(L.entry(0, i0) & ~RF_PARTIAL_BIT) : 0x7fffffff;
+    const int e1 = i1 < L.n1 ? (int)(L.entry(1, i1) & ~RF_PARTIAL_BIT) : 0x7fffffff;
+    tile = min(e0, e1);
+    if (tile == 0x7fffffff) return false;
+    uses = (e0 == tile ? 1 : 0) | (e1 == tile ? 2 : 0);
+    i0 += e0 == tile;
+    i1 += e1 == tile;
+    return true;
+  }
+};
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_constant__ Maps maps, const RfAttnArgs a) {
-  using L = Smem<D>;
-  constexpr int KB = L::KB;
-  constexpr uint32_t TILE_BYTES = KB * L::BLK;
-  constexpr uint32_t TMEM_COLS = 256;          // S: columns [0,128), O tile: [128, 128+D)
-  constexpr uint32_t S_COL = 0, O_COL = 128;
+  using C = Cfg<D>;
+  constexpr int KB = C::KB;
   constexpr uint32_t IDESC_S = idesc_bf16(BM, BN, 0);
   constexpr uint32_t IDESC_PV = idesc_bf16(BM, D, 1);
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t bar_q = base + L::BAR, bar_kv0 = bar_q + 8, bar_mma = bar_q + 24;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::MISC);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::MISC + 8);
+  auto bar = [&](int slot) -> uint32_t { return base + C::BAR + 8u * slot; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + C::MISC);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::MISC + 8);
 
   const RfGeom& g = a.g;
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int qt = blockIdx.x, bh = blockIdx.y;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.y;
+  const int qt0 = 2 * blockIdx.x, qt1 = qt0 + 1;
 
   int cls = RF_DENSE;
   if (a.head_class != nullptr) {
@@ -109,186 +158,257 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   const CUtensorMap* map_q = &maps.m[perm ? 3 : 0];
   const CUtensorMap* map_k = &maps.m[perm ? 4 : (tex ? 6 : 1)];
   const CUtensorMap* map_v = &maps.m[perm ? 5 : (tex ? 7 : 2)];
-  const int lkv = rf_kv_len(g, cls);
-  const bool listed = a.head_class != nullptr;
-  const int n_tiles = listed ? a.count[(size_t)bh * g.nQ + qt] : rf_cdiv(lkv, BN);
-  const int32_t* list = listed ? a.kv_tile + ((size_t)bh * g.nQ + qt) * g.nKmax : nullptr;
+
+  Lists L;
+  L.lkv = rf_kv_len(g, cls);
+  L.listed = a.head_class != nullptr;
+  if (L.listed) {
+    L.n0 = a.count[(size_t)bh * g.nQ + qt0];
+    L.n1 = qt1 < g.nQ ? a.count[(size_t)bh * g.nQ + qt1] : 0;
+    L.l0 = a.kv_tile + ((size_t)bh * g.nQ + qt0) * g.nKmax;
+    L.l1 = a.kv_tile + ((size_t)bh * g.nQ + min(qt1, g.nQ - 1)) * g.nKmax;
+  } else {
+    L.n0 = rf_cdiv(L.lkv, BN);
+    L.n1 = qt1 < g.nQ ? L.n0 : 0;
+    L.l0 = L.l1 = nullptr;
+  }
 
   if (tid == 0) {
-    mbar_init(bar_q, 1);
-    mbar_init(bar_kv0, 1);
-    mbar_init(bar_kv0 + 8, 1);
-    mbar_init(bar_mma, 1);
+    mbar_init(bar(C::B_Q), 1);
+    for (int s = 0; s < C::NK; ++s) { mbar_init(bar(C::B_KF + s), 1); mbar_init(bar(C::B_KE + s), 1); }
+    for (int s = 0; s < C::NV; ++s) { mbar_init(bar(C::B_VF + s), 1); mbar_init(bar(C::B_VE + s), 1); }
+    for (int j = 0; j < 2; ++j) {
+      mbar_init(bar(C::B_SF + j), 1);
+      mbar_init(bar(C::B_PF + j), 4);   // one arrival per softmax warp
+      mbar_init(bar(C::B_OF + j), 1);
+    }
     *abort_flag = 0;
     mbar_init_fence();
-    prefetch_tmap(map_q);
-    prefetch_tmap(map_k);
-    prefetch_tmap(map_v);
   }
-  if (warp == 0) {
+  if (warp == kTmaWarp) {
+    if (lane == 0) { prefetch_tmap(map_q); prefetch_tmap(map_k); prefetch_tmap(map_v); }
     __syncwarp();
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS);
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
   const WaitCtx wc{abort_flag, a.dev_status};
 
-  auto tile_entry = [&](int i) -> uint32_t {
-    if (listed) return (uint32_t)list[i];
-    const bool tail = (i + 1) * BN > lkv;
-    return (uint32_t)i | (tail ? RF_PARTIAL_BIT : 0u);
-  };
-  auto load_kv = [&](int i, int stage) {
-    const int tile = (int)(tile_entry(i) & ~RF_PARTIAL_BIT);
-    const uint32_t bar = bar_kv0 + 8 * stage;
-    mbar_expect_tx(bar, 2 * TILE_BYTES);
+  if (warp == kTmaWarp) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(bar(C::B_Q), 2 * C::TILE);
 #pragma unroll
-    for (int kb = 0; kb < KB; ++kb) {
-      tma_load_3d(base + L::K0 + stage * TILE_BYTES + kb * L::BLK, map_k, kb * 64, tile * BN, bh, bar);
-      tma_load_3d(base + L::V0 + stage * TILE_BYTES + kb * L::BLK, map_v, kb * 64, tile * BN, bh, bar);
-    }
-  };
-
-  if (tid == 0) {
-    mbar_expect_tx(bar_q, TILE_BYTES);
+      for (int j = 0; j < 2; ++j)
 #pragma unroll
-    for (int kb = 0; kb < KB; ++kb) tma_load_3d(base + L::Q + kb * L::BLK, map_q, kb * 64, qt * BM, bh, bar_q);
-    if (n_tiles > 0) load_kv(0, 0);
-  }
-
-  const int r = qt * BM + tid;                       // this thread's query slot
-  const RowMask rmask = make_row_mask(g, cls, min(r, g.N - 1));
-  float o_acc[D];
+        for (int kb = 0; kb < KB; ++kb)
+          tma_load_3d(base + C::Q + j * C::TILE + kb * C::BLK, map_q, kb * 64, (qt0 + j) * BM, bh, bar(C::B_Q));
+      Merge mg;
+      int tile, uses;
+      for (int u = 0; mg.next(L, tile, uses); ++u) {
+        const int ks = u % C::NK, vs = u % C::NV;
+        if (u >= C::NK) mbar_wait(bar(C::B_KE + ks), ((u / C::NK) - 1) & 1, wc);
+        mbar_expect_tx(bar(C::B_KF + ks), C::TILE);
 #pragma unroll
-  for (int d = 0; d < D; ++d) o_acc[d] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f;
-  const float sc = a.scale_log2;
-
-  for (int it = 0; it < n_tiles; ++it) {
-    const int st = it & 1;
-    const uint32_t entry = tile_entry(it);
-    const bool partial = (entry & RF_PARTIAL_BIT) != 0;
-    const int u0 = (int)(entry & ~RF_PARTIAL_BIT) * BN;
-
-    if (tid == 0) {
-      if (it + 1 < n_tiles) load_kv(it + 1, st ^ 1);
-      if (it == 0) mbar_wait(bar_q, 0, wc);
-      mbar_wait(bar_kv0 + 8 * st, (it >> 1) & 1, wc);
-      tc_fence_after();
+        for (int kb = 0; kb < KB; ++kb)
+          tma_load_3d(base + C::K0 + ks * C::TILE + kb * C::BLK, map_k, kb * 64, tile * BN, bh, bar(C::B_KF + ks));
+        if (u >= C::NV) mbar_wait(bar(C::B_VE + vs), ((u / C::NV) - 1) & 1, wc);
+        mbar_expect_tx(bar(C::B_VF + vs), C::TILE);
 #pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) {
-        const uint32_t off = (ks >> 2) * L::BLK + (ks & 3) * 32;
-        mma_ss(tmem_base + S_COL, smem_desc_sw128(base + L::Q + off, 16, 1024),
-               smem_desc_sw128(base + L::K0 + st * TILE_BYTES + off, 16, 1024), IDESC_S, ks > 0);
+        for (int kb = 0; kb < KB; ++kb)
+          tma_load_3d(base + C::V0 + vs * C::TILE + kb * C::BLK, map_v, kb * 64, tile * BN, bh, bar(C::B_VF + vs));
       }
-      tc_commit(bar_mma);
     }
-    __syncwarp();
-    mbar_wait(bar_mma, 0, wc);
-    tc_fence_after();
-
-    // pass 1: row maximum of the scaled, masked scores
-    float rmax = -INFINITY;
+  } else if (warp == kMmaWarp) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      auto issue_s = [&](int j, int ks) {
 #pragma unroll
-    for (int c = 0; c < BN / 32; ++c) {
-      uint32_t v[32];
-      tmem_ld32(tmem_lane + S_COL + c * 32, v);
-      tc_wait_ld();
+        for (int k = 0; k < D / 16; ++k) {
+          const uint32_t off = (k >> 2) * C::BLK + (k & 3) * 32;
+          mma_ss(tmem_base + (j ? C::S_COL1 : C::S_COL0), smem_desc_sw128(base + C::Q + j * C::TILE + off, 16, 1024),
+                 smem_desc_sw128(base + C::K0 + ks * C::TILE + off, 16, 1024), IDESC_S, k > 0);
+        }
+        tc_commit(bar(C::B_SF + j));
+      };
+      auto issue_pv = [&](int j, int vs, bool first) {
+#pragma unroll
+        for (int k = 0; k < BN / 16; ++k) {
+          mma_ts(tmem_base + (j ? C::O_COL1 : C::O_COL0), tmem_base + (j ? C::S_COL1 : C::S_COL0) + k * 8,
+                 smem_desc_sw128(base + C::V0 + vs * C::TILE + k * 2048, C::BLK, 1024), IDESC_PV, (!first) || k > 0);
+        }
+        tc_commit(bar(C::B_OF + j));
+      };
+      Merge mg;
+      int cur_tile, cur_uses, nxt_tile = 0, nxt_uses = 0;
+      bool has_cur = mg.next(L, cur_tile, cur_uses);
+      int pv_cnt[2] = {0, 0};
+      mbar_wait(bar(C::B_Q), 0, wc);
+      if (has_cur) {
+        mbar_wait(bar(C::B_KF + 0), 0, wc);
+        tc_fence_after();
+        if (cur_uses & 1) issue_s(0, 0);
+        if (cur_uses & 2) issue_s(1, 0);
+        tc_commit(bar(C::B_KE + 0));
+      }
+      for (int u = 0; has_cur; ++u) {
+        const bool has_nxt = mg.next(L, nxt_tile, nxt_uses);
+        const int vs = u % C::NV, ksn = (u + 1) % C::NK;
+        bool v_ready = false, k_ready = false;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          if (cur_uses & (1 << j)) {
+            mbar_wait(bar(C::B_PF + j), pv_cnt[j] & 1, wc);
+            if (!v_ready) { mbar_wait(bar(C::B_VF + vs), (u / C::NV) & 1, wc); v_ready = true; }
+            tc_fence_after();
+            issue_pv(j, vs, pv_cnt[j] == 0);
+            ++pv_cnt[j];
+          }
+          if (has_nxt && (nxt_uses & (1 << j))) {
+            if (!k_ready) { mbar_wait(bar(C::B_KF + ksn), ((u + 1) / C::NK) & 1, wc); k_ready = true; }
+            tc_fence_after();
+            issue_s(j, ksn);
+          }
+        }
+        tc_commit(bar(C::B_VE + vs));
+        if (has_nxt) tc_commit(bar(C::B_KE + ksn));
+        has_cur = has_nxt;
+        cur_tile = nxt_tile;
+        cur_uses = nxt_uses;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax + epilogue, one thread per query row
+    const int j = warp >> 2;                       // stream
+    const int row_in_tile = tid & 127;
+    const int r = (qt0 + j) * BM + row_in_tile;    // query slot in the head's coordinate space
+    const int n = j == 0 ? L.n0 : L.n1;
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t t_s = tmem_base + lane_sel + (j ? C::S_COL1 : C::S_COL0);
+    const uint32_t t_o = tmem_base + lane_sel + (j ? C::O_COL1 : C::O_COL0);
+    const RowMask rmask = make_row_mask(g, cls, min(r, g.N - 1));
+    const float sc = a.scale_log2;
+    float m_run = -INFINITY;   // running maximum, log2 domain (score * sc)
+    float l_run = 0.f;
+
+    for (int it = 0; it < n; ++it) {
+      const uint32_t entry = L.entry(j, it);
+      const bool partial = (entry & RF_PARTIAL_BIT) != 0;
+      const int u0 = (int)(entry & ~RF_PARTIAL_BIT) * BN;
+      mbar_wait(bar(C::B_SF + j), it & 1, wc);
+      tc_fence_after();
+      uint32_t s[128];
+      {
+        uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+        uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+        uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+        uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+        tmem_ld32(t_s, s0);
+        tmem_ld32(t_s + 32, s1);
+        tmem_ld32(t_s + 64, s2);
+        tmem_ld32(t_s + 96, s3);
+        tc_wait_ld();
+      }
       if (partial) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (rmask.keep(u0 + c * 32 + j)) rmax = fmaxf(rmax, __uint_as_float(v[j]) * sc);
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) rmax = fmaxf(rmax, __uint_as_float(v[j]) * sc);
+        for (int c = 0; c < 128; ++c)
+          if (!rmask.keep(u0 + c)) s[c] = 0xff800000u;  // -inf
       }
-    }
-    const float m_new = fmaxf(m_run, rmax);
-    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-    const float alpha = exp2f(m_run - m_use);
-    m_run = m_new;
-    l_run *= alpha;
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-    for (int d = 0; d < D; ++d) o_acc[d] *= alpha;
+      for (int c = 0; c < 128; c += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(s[c]));
+        mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
+        mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+      }
+      const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc;
 
-    // pass 2: P = exp2(S*scale - m), row sum, bf16 P into swizzled shared memory (K-major A operand)
-#pragma unroll
-    for (int c = 0; c < BN / 32; ++c) {
-      uint32_t v[32];
-      tmem_ld32(tmem_lane + S_COL + c * 32, v);
-      tc_wait_ld();
-      float p[32];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        float e = exp2f(fmaf(__uint_as_float(v[j]), sc, -m_use));
-        if (partial && !rmask.keep(u0 + c * 32 + j)) e = 0.f;
-        p[j] = e;
-        l_run += e;
+      // raise the running maximum only when it grows by more than the threshold
+      const bool raise = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
+      float alpha = 1.f;
+      if (raise) {
+        alpha = ex2(m_run - m_tile);   // 0 when m_run = -inf
+        m_run = m_tile;
+        l_run *= alpha;
       }
-      const uint32_t prow = base + L::P + (c >> 1) * L::BLK + tid * 128;
+      if (it > 0 && __any_sync(0xffffffffu, raise)) {
+        // O of the previous tiles must be complete before it is rescaled
+        mbar_wait(bar(C::B_OF + j), (it - 1) & 1, wc);
+        tc_fence_after();
 #pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        const uint32_t chunk = (uint32_t)((c & 1) * 4 + jj) ^ (uint32_t)(tid & 7);
-        const uint32_t w0 = pack_bf16(p[jj * 8 + 0], p[jj * 8 + 1]), w1 = pack_bf16(p[jj * 8 + 2], p[jj * 8 + 3]);
-        const uint32_t w2 = pack_bf16(p[jj * 8 + 4], p[jj * 8 + 5]), w3 = pack_bf16(p[jj * 8 + 6], p[jj * 8 + 7]);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(prow + (chunk << 4)), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_o + c * 32, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+          tmem_st32(t_o + c * 32, v);
+        }
+        tc_wait_st();
       }
+      const float m_use = m_run == -INFINITY ? 0.f : m_run;
+      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+      uint32_t pk[64];
+#pragma unroll
+      for (int c = 0; c < 128; c += 4) {
+        const float p0 = ex2(fmaf(__uint_as_float(s[c]), sc, -m_use));
+        const float p1 = ex2(fmaf(__uint_as_float(s[c + 1]), sc, -m_use));
+        const float p2 = ex2(fmaf(__uint_as_float(s[c + 2]), sc, -m_use));
+        const float p3 = ex2(fmaf(__uint_as_float(s[c + 3]), sc, -m_use));
+        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+        pk[c / 2] = pack_bf16(p0, p1);
+        pk[c / 2 + 1] = pack_bf16(p2, p3);
+      }
+      l_run += (l0 + l1) + (l2 + l3);
+      {
+        uint32_t(&p0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[0]);
+        uint32_t(&p1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[32]);
+        tmem_st32(t_s, p0);
+        tmem_st32(t_s + 32, p1);
+        tc_wait_st();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(C::B_PF + j));
     }
-    fence_proxy_async_smem();
-    tc_fence_before();
-    __syncthreads();
 
-    if (tid == 0) {
+    if (n > 0) {
+      mbar_wait(bar(C::B_OF + j), (n - 1) & 1, wc);
       tc_fence_after();
+      int tok = r;
+      if (perm && r < g.Nv) tok = (r % g.T) * g.S + r / g.T;
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      uint4* dst = reinterpret_cast<uint4*>(a.o + ((size_t)bh * g.N + min(tok, g.N - 1)) * D);
 #pragma unroll
-      for (int ks = 0; ks < BN / 16; ++ks) {
-        const uint32_t poff = (ks >> 2) * L::BLK + (ks & 3) * 32;
-        mma_ss(tmem_base + O_COL, smem_desc_sw128(base + L::P + poff, 16, 1024),
-               smem_desc_sw128(base + L::V0 + st * TILE_BYTES + ks * 2048, L::BLK, 1024), IDESC_PV, ks > 0);
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld32(t_o + c * 32, v);   // warp-collective: rows past N take part, they just do not store
+        tc_wait_ld();
+        if (r < g.N) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(v[i + 4]) * inv, __uint_as_float(v[i + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(v[i + 6]) * inv, __uint_as_float(v[i + 7]) * inv);
+            dst[(c * 32 + i) / 8] = w;
+          }
+        }
       }
-      tc_commit(bar_mma);
-    }
-    __syncwarp();
-    mbar_wait(bar_mma, 1, wc);
-    tc_fence_after();
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t v[32];
-      tmem_ld32(tmem_lane + O_COL + c * 32, v);
-      tc_wait_ld();
-#pragma unroll
-      for (int j = 0; j < 32; ++j) o_acc[c * 32 + j] += __uint_as_float(v[j]);
+      if (r < g.N && a.lse != nullptr) a.lse[(size_t)bh * g.N + tok] = (m_run + log2f(l_run)) * 0.6931471805599453f;
     }
   }
 
-  // epilogue: normalise, write O (original token order) and lse
-  if (r < g.N) {
-    int tok = r;
-    if (perm && r < g.Nv) tok = (r % g.T) * g.S + r / g.T;
-    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-    uint4* dst = reinterpret_cast<uint4*>(a.o + ((size_t)bh * g.N + tok) * D);
-#pragma unroll
-    for (int d = 0; d < D; d += 8) {
-      uint4 w;
-      w.x = pack_bf16(o_acc[d] * inv, o_acc[d + 1] * inv);
-      w.y = pack_bf16(o_acc[d + 2] * inv, o_acc[d + 3] * inv);
-      w.z = pack_bf16(o_acc[d + 4] * inv, o_acc[d + 5] * inv);
-      w.w = pack_bf16(o_acc[d + 6] * inv, o_acc[d + 7] * inv);
-      dst[d / 8] = w;
-    }
-    if (a.lse != nullptr) a.lse[(size_t)bh * g.N + tok] = (m_run + log2f(l_run)) * 0.6931471805599453f;
-  }
-
-  // never leave with a TMA still in flight: the Q load (unused when the list is empty)
-  if (tid == 0 && n_tiles == 0) mbar_wait(bar_q, 0, wc);
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == kTmaWarp) {
+    if (*abort_flag) __nanosleep(20000);  // let abandoned copies land before shared memory is released
     __syncwarp();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
@@ -298,14 +418,14 @@ rf_status launch(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st) 
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return RF_ERR_CUDA;
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(rf_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem<D>::ALLOC) != cudaSuccess)
+    if (cudaFuncSetAttribute(rf_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<D>::ALLOC) != cudaSuccess)
       return RF_ERR_CUDA;
     configured[dev] = true;
   }
   Maps m;
   for (int i = 0; i < 8; ++i) m.m[i] = maps[i];
-  dim3 grid(a.g.nQ, a.g.B * a.g.H);
-  rf_attn_kernel<D><<<grid, kThreads, Smem<D>::ALLOC, st>>>(m, a);
+  dim3 grid(rf_cdiv(a.g.nQ, 2), a.g.B * a.g.H);
+  rf_attn_kernel<D><<<grid, kThreads, Cfg<D>::ALLOC, st>>>(m, a);
   return cudaGetLastError() == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }
 

@@ -7,6 +7,7 @@
 //   warps 4-7  softmax of stream 1
 //   warp  8    TMA producer: Q once, then K and V tiles into two shared-memory rings
 //   warp  9    MMA issuer: tcgen05.mma, accumulators in TMEM (S0, S1, O0, O1)
+//   (warps 10-11 only fill the third warpgroup, which hands its registers to the softmax warpgroups)
 // Per listed tile and stream: S lands in TMEM, the softmax warps read their rows (tcgen05.ld), keep a
 // running maximum and sum in fp32, write P as packed bf16 back into the S columns (tcgen05.st) and the
 // MMA warp multiplies it with V straight from TMEM.  The running maximum is only raised when it grows
@@ -20,8 +21,7 @@ namespace {
 using namespace sm100;
 
 constexpr int BM = 128, BN = 128;
-constexpr int kSoftmaxThreads = 256;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;               // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
 constexpr int kTmaWarp = 8, kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
@@ -54,21 +54,41 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// Element mask of one query row in the head's key-slot space.
+// Element mask of one query row in the head's key-slot space, evaluated per tile as a 128-bit word
+// (bit c = key slot u0 + c kept).  Every pattern's kept set is a union of a few slot intervals:
+// one window [lo, hi) (Spatial, position-major Temporal), one band per frame (Temporal in original
+// order) and the always-kept text slots [text0, lkv).  Kept compact on purpose: PARTIAL tiles are
+// rare, and a large rarely-run code block costs more in instruction fetch than in arithmetic.
 struct RowMask {
   int lo, hi;        // kept video slots [lo, hi) when !periodic
   int text0;         // first always-kept (text) slot
   int lkv;           // number of key slots
-  int p, ws, S;      // periodic form: |slot % S - p| <= ws
+  int p, ws, S, T;   // periodic form: |slot % S - p| <= ws for slots of frames 0..T-1
   bool periodic;
-  __device__ __forceinline__ bool keep(int u) const {
-    if (u >= lkv) return false;
-    if (u >= text0) return true;
-    if (periodic) {
-      const int d = (u % S) - p;
-      return (d < 0 ? -d : d) <= ws;
+
+  static __device__ __forceinline__ uint32_t below(int n) {  // bits [0, n) set, n in [0, 32]
+    return n >= 32 ? 0xffffffffu : ((1u << n) - 1u);
+  }
+  // OR the slots [a, b) (absolute) into the tile's words.
+  static __device__ __forceinline__ void add(uint32_t (&w)[4], int u0, int a, int b) {
+    a = max(a - u0, 0);
+    b = min(b - u0, BN);
+    if (a >= b) return;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int lo_k = min(max(a - 32 * k, 0), 32), hi_k = min(max(b - 32 * k, 0), 32);
+      w[k] |= below(hi_k) & ~below(lo_k);
     }
-    return u >= lo && u < hi;
+  }
+  __device__ __noinline__ void tile_bits(int u0, uint32_t (&w)[4]) const {
+    w[0] = w[1] = w[2] = w[3] = 0u;
+    if (periodic) {
+      const int f1 = min((u0 + BN - 1) / S, T - 1);
+      for (int f = u0 / S; f <= f1; ++f) add(w, u0, f * S + max(p - ws, 0), f * S + min(p + ws, S - 1) + 1);
+    } else {
+      add(w, u0, lo, min(hi, text0));
+    }
+    add(w, u0, text0, lkv);
   }
 };
 
@@ -78,7 +98,7 @@ __device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r
   m.text0 = m.lkv;
   m.lo = 0;
   m.hi = m.lkv;
-  m.p = 0; m.ws = g.ws; m.S = g.S;
+  m.p = 0; m.ws = g.ws; m.S = g.S; m.T = g.T;
   m.periodic = false;
   if ((cls == RF_SPATIAL || cls == RF_TEMPORAL) && r < g.Nv) {
     m.text0 = g.Nv;
@@ -196,6 +216,8 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   const uint32_t tmem_base = *tmem_slot;
   const WaitCtx wc{abort_flag, a.dev_status};
 
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -279,7 +301,9 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         cur_uses = nxt_uses;
       }
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ------------------------------------------------------------ softmax + epilogue, one thread per query row
     const int j = warp >> 2;                       // stream
     const int row_in_tile = tid & 127;
@@ -312,9 +336,11 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         tc_wait_ld();
       }
       if (partial) {
+        uint32_t w[4];
+        rmask.tile_bits(u0, w);
 #pragma unroll
         for (int c = 0; c < 128; ++c)
-          if (!rmask.keep(u0 + c)) s[c] = 0xff800000u;  // -inf
+          if (!((w[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf
       }
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll

@@ -20,7 +20,7 @@
  *   - Host-detectable errors return a code before anything is launched.  Device-detected ones
  *     (a bounded wait that ran out, a head class outside 0..3) are written to *dev_status
  *     (device int32, may be NULL; never reset by the library) and the kernels still terminate.
- *   - Supported: D in {64, 128}; block_m = block_n = 128 for the attention entry points;
+ *   - Supported: D in {64, 96, 128}; block_m = block_n = 128 for the attention entry points;
  *     rf_build_block_mask alone accepts any power-of-two blocks >= 16.
  */
 #ifndef RAINFUSION_H_

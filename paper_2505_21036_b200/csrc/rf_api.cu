@@ -95,7 +95,7 @@ bool encode_map(CUtensorMap* m, const void* ptr, int D, int rows, int head_rows,
 rf_status check_attn_shape(const rf_shape* s) {
   rf_status st = check_shape(s);
   if (st != RF_OK) return st;
-  if (s->D != 64 && s->D != 128) return RF_ERR_UNSUPPORTED;
+  if (s->D != 64 && s->D != 96 && s->D != 128) return RF_ERR_UNSUPPORTED;
   return RF_OK;
 }
 

@@ -29,11 +29,17 @@ struct Maps { CUtensorMap m[8]; };
 
 template <int D>
 struct Cfg {
-  static constexpr int KB = D / 64;                   // 64-column (128-byte) blocks per row
+  static constexpr int KB = (D + 63) / 64;            // 64-column (128-byte) blocks per row
+  // first column of block kb: D = 96 is held as two overlapping 64-column blocks, [0,64) and [32,96)
+  static constexpr int COL1 = D - 64;
   static constexpr uint32_t BLK = 128 * 128;          // bytes of one 128-row x 64-col bf16 block
   static constexpr uint32_t TILE = KB * BLK;          // bytes of one 128-row tile
-  static constexpr int NK = D == 128 ? 2 : 4;         // K ring depth
-  static constexpr int NV = D == 128 ? 2 : 4;         // V ring depth
+  static constexpr int NK = D == 64 ? 4 : 2;          // K ring depth
+  static constexpr int NV = D == 64 ? 4 : 2;          // V ring depth
+  // byte offset, inside a tile, of the 16 columns of k-step ks of the Q K^T contraction
+  static __host__ __device__ constexpr uint32_t koff(int ks) {
+    return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks * 16 - COL1) * 2u;
+  }
   static constexpr uint32_t Q = 0;
   static constexpr uint32_t K0 = Q + 2 * TILE;
   static constexpr uint32_t V0 = K0 + NK * TILE;
@@ -151,7 +157,8 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   using C = Cfg<D>;
   constexpr int KB = C::KB;
   constexpr uint32_t IDESC_S = idesc_bf16(BM, BN, 0);
-  constexpr uint32_t IDESC_PV = idesc_bf16(BM, D, 1);
+  constexpr uint32_t IDESC_PV = idesc_bf16(BM, D == 96 ? 64 : D, 1);
+  constexpr uint32_t IDESC_PV32 = idesc_bf16(BM, 32, 1);   // D = 96: columns [64, 96) of O
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -226,7 +233,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       for (int j = 0; j < 2; ++j)
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_3d(base + C::Q + j * C::TILE + kb * C::BLK, map_q, kb * 64, (qt0 + j) * BM, bh, bar(C::B_Q));
+          tma_load_3d(base + C::Q + j * C::TILE + kb * C::BLK, map_q, kb * C::COL1, (qt0 + j) * BM, bh, bar(C::B_Q));
       Merge mg;
       int tile, uses;
       for (int u = 0; mg.next(L, tile, uses); ++u) {
@@ -235,12 +242,12 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         mbar_expect_tx(bar(C::B_KF + ks), C::TILE);
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_3d(base + C::K0 + ks * C::TILE + kb * C::BLK, map_k, kb * 64, tile * BN, bh, bar(C::B_KF + ks));
+          tma_load_3d(base + C::K0 + ks * C::TILE + kb * C::BLK, map_k, kb * C::COL1, tile * BN, bh, bar(C::B_KF + ks));
         if (u >= C::NV) mbar_wait(bar(C::B_VE + vs), ((u / C::NV) - 1) & 1, wc);
         mbar_expect_tx(bar(C::B_VF + vs), C::TILE);
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_3d(base + C::V0 + vs * C::TILE + kb * C::BLK, map_v, kb * 64, tile * BN, bh, bar(C::B_VF + vs));
+          tma_load_3d(base + C::V0 + vs * C::TILE + kb * C::BLK, map_v, kb * C::COL1, tile * BN, bh, bar(C::B_VF + vs));
       }
     }
   } else if (warp == kMmaWarp) {
@@ -249,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       auto issue_s = [&](int j, int ks) {
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = (k >> 2) * C::BLK + (k & 3) * 32;
+          const uint32_t off = C::koff(k);
           mma_ss(tmem_base + (j ? C::S_COL1 : C::S_COL0), smem_desc_sw128(base + C::Q + j * C::TILE + off, 16, 1024),
                  smem_desc_sw128(base + C::K0 + ks * C::TILE + off, 16, 1024), IDESC_S, k > 0);
         }
@@ -260,6 +267,10 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         for (int k = 0; k < BN / 16; ++k) {
           mma_ts(tmem_base + (j ? C::O_COL1 : C::O_COL0), tmem_base + (j ? C::S_COL1 : C::S_COL0) + k * 8,
                  smem_desc_sw128(base + C::V0 + vs * C::TILE + k * 2048, C::BLK, 1024), IDESC_PV, (!first) || k > 0);
+          if (D == 96)  // columns [64, 96): the upper half of the second block's 128-byte rows
+            mma_ts(tmem_base + (j ? C::O_COL1 : C::O_COL0) + 64, tmem_base + (j ? C::S_COL1 : C::S_COL0) + k * 8,
+                   smem_desc_sw128(base + C::V0 + vs * C::TILE + C::BLK + k * 2048 + 64, C::BLK, 1024), IDESC_PV32,
+                   (!first) || k > 0);
         }
         tc_commit(bar(C::B_OF + j));
       };
@@ -460,6 +471,7 @@ rf_status launch(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st) 
 rf_status rf_launch_attention(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st) {
   switch (a.g.D) {
     case 64: return launch<64>(a, maps, st);
+    case 96: return launch<96>(a, maps, st);
     case 128: return launch<128>(a, maps, st);
   }
   return RF_ERR_UNSUPPORTED;

@@ -39,7 +39,8 @@ typedef enum {
   RF_ERR_UNSUPPORTED = 2,
   RF_ERR_WORKSPACE_TOO_SMALL = 3,
   RF_ERR_CUDA = 4,
-  RF_ERR_TIMEOUT = 5
+  RF_ERR_TIMEOUT = 5,
+  RF_ERR_STATIC_SCRATCH_TOO_SMALL = 6
 } rf_status;
 
 /* Head categories (Sec. 3.2).  RF_DENSE is not an ARM outcome; a caller may force it. */
@@ -141,6 +142,32 @@ rf_status rf_reorder_tokens(const rf_shape *shape, const rf_params *params, cons
 /* Full 3D attention (Eq. 1-2, all-zero mask): the same kernel walking every tile.  ws may be NULL. */
 rf_status rf_dense_attn_fwd(const rf_shape *shape, const void *q, const void *k, const void *v, void *o,
                             float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
+
+/*
+ * rf_arm_classify for callers that cannot provide a workspace.  (The paper has no counterpart: this is
+ * a packaging variant of rf_arm_classify, same kernels, same results.)
+ *
+ * Some callers of this library run where device allocation is off limits: inside a serving loop
+ * whose memory pool was sized and frozen at start-up, or under a framework allocator that must not be
+ * re-entered from a plug-in, so they have no buffer to hand over as `ws` and may not call cudaMalloc
+ * to make one.  This entry point takes only inputs and outputs.  Its per-row recall scratch lives in
+ * a fixed array inside the library's device image: RF_ARM_STATIC_SCRATCH_FLOATS floats (4 MiB) that
+ * every GPU which loads the library holds until the process exits.
+ *
+ *   - Limit: 2 * B * H * 3 * roundup64(max(frame_h*frame_w, ceil(T*frame_h*frame_w / sample_stride)))
+ *     floats must fit (the HunyuanVideo-720p layer needs 525 312).  Larger problems are rejected
+ *     with RF_ERR_STATIC_SCRATCH_TOO_SMALL before anything is launched.
+ *   - Allocates nothing: no cudaMalloc / cudaFree, no allocating library call.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current).  Make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to
+ *     start at zero (every element that is read was written earlier in the same call), but two calls
+ *     that overlap on the GPU - different streams, or different host threads - race on it.  Serialise
+ *     them, or use rf_arm_classify with separate workspaces.
+ */
+#define RF_ARM_STATIC_SCRATCH_FLOATS (1u << 20)
+rf_status rf_arm_classify_noalloc(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
+                                  int32_t *head_class, float *recall, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -18,7 +18,8 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librainfus
 _lib = None
 
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
-           "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd"]
+           "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
+           "rf_arm_classify_noalloc"]
 
 
 class rf_shape(C.Structure):
@@ -61,6 +62,8 @@ def load():
     lib.rf_workspace_bytes.argtypes = [P(rf_shape), P(rf_params)]
     lib.rf_arm_classify.restype = I
     lib.rf_arm_classify.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, Z, V]
+    lib.rf_arm_classify_noalloc.restype = I
+    lib.rf_arm_classify_noalloc.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V]
     lib.rf_build_block_mask.restype = I
     lib.rf_build_block_mask.argtypes = [P(rf_shape), P(rf_params), V, P(rf_schedule), V, V]
     lib.rf_sparse_attn_fwd.restype = I
@@ -146,6 +149,15 @@ def alloc_workspace(shape: rf_shape, params: rf_params, device):
 def rf_arm_classify(shape, params, q, k, head_class, recall, ws):
     _check(load().rf_arm_classify(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), head_class.data_ptr(),
                                   _ptr(recall), ws.data_ptr(), ws.numel(), _stream()), "rf_arm_classify")
+
+
+def rf_arm_classify_noalloc(shape, params, q, k, head_class, recall):
+    """rf_arm_classify without a workspace: for callers that may not allocate device memory (a frozen
+    serving pool, a plug-in that must not re-enter the framework allocator).  The scratch is a fixed
+    4 MiB array inside the library; problems that need more raise RainFusionError.  Calls that overlap
+    on the GPU share that array and race; run them one after the other."""
+    _check(load().rf_arm_classify_noalloc(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(),
+                                          head_class.data_ptr(), _ptr(recall), _stream()), "rf_arm_classify_noalloc")
 
 
 def rf_build_block_mask(shape, params, head_class, sched: Schedule, dev_status=None):

@@ -101,6 +101,15 @@ rf_status check_attn_shape(const rf_shape* s) {
 
 }  // namespace
 
+rf_status rf_checked_geom(const rf_shape* shape, const rf_params* params, RfGeom* out) {
+  rf_status st = check_shape(shape);
+  if (st != RF_OK) return st;
+  st = check_params(params);
+  if (st != RF_OK) return st;
+  *out = make_geom(shape, params);
+  return RF_OK;
+}
+
 extern "C" {
 
 const char* rf_status_string(rf_status s) {
@@ -111,6 +120,8 @@ const char* rf_status_string(rf_status s) {
     case RF_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case RF_ERR_CUDA: return "CUDA error";
     case RF_ERR_TIMEOUT: return "device-side wait timed out";
+    case RF_ERR_STATIC_SCRATCH_TOO_SMALL:
+      return "problem needs more scratch than the library's built-in array holds (use the workspace entry point)";
   }
   return "unknown status";
 }

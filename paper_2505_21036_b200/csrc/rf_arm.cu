@@ -254,3 +254,47 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
                                                   head_class, recall);
   return cudaGetLastError();
 }
+
+// ------------------------------------------------------------------------------------------------
+// Entry point for callers that can neither pass a workspace nor allocate one: the per-row recall
+// scratch is a fixed array in this library's device image.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) float g_arm_static_scratch[RF_ARM_STATIC_SCRATCH_FLOATS];
+
+namespace {
+// Device address of g_arm_static_scratch per device.  In host code the array's name is only a
+// handle for the runtime, not a pointer a kernel may use; the address comes from cudaGetSymbolAddress
+// with the device in question current.
+float* static_scratch_ptr(int dev, cudaError_t* err) {
+  static float* ptrs[64] = {};
+  *err = cudaSuccess;
+  if (dev < 0 || dev >= 64) { *err = cudaErrorInvalidDevice; return nullptr; }
+  if (ptrs[dev] == nullptr) {
+    void* p = nullptr;
+    *err = cudaGetSymbolAddress(&p, g_arm_static_scratch);
+    if (*err != cudaSuccess) return nullptr;
+    ptrs[dev] = static_cast<float*>(p);
+  }
+  return ptrs[dev];
+}
+}  // namespace
+
+extern "C" rf_status rf_arm_classify_noalloc(const rf_shape* shape, const rf_params* params, const void* q,
+                                             const void* k, int32_t* head_class, float* recall, void* cuda_stream) {
+  RfGeom g;
+  rf_status st = rf_checked_geom(shape, params, &g);
+  if (st != RF_OK) return st;
+  if (g.D != 64 && g.D != 96 && g.D != 128) return RF_ERR_UNSUPPORTED;
+  if (q == nullptr || k == nullptr || head_class == nullptr) return RF_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) & 15u) != 0 || (reinterpret_cast<uintptr_t>(k) & 15u) != 0) return RF_ERR_INVALID_ARG;
+  if (rf_arm_scratch_floats(g, params->sample_stride) > (size_t)RF_ARM_STATIC_SCRATCH_FLOATS)
+    return RF_ERR_STATIC_SCRATCH_TOO_SMALL;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RF_ERR_CUDA;
+  cudaError_t e;
+  float* scratch = static_scratch_ptr(dev, &e);
+  if (scratch == nullptr) return RF_ERR_CUDA;
+  e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, static_cast<const __nv_bfloat16*>(q),
+                    static_cast<const __nv_bfloat16*>(k), head_class, recall, scratch, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
+}

@@ -44,6 +44,8 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
                           const __nv_bfloat16* k, int32_t* head_class, float* recall, float* row_scratch,
                           cudaStream_t st);
 size_t rf_arm_scratch_floats(const RfGeom& g, int omega);
+// Validates shape and parameters as the entry points do and fills the kernel-side geometry.
+rf_status rf_checked_geom(const rf_shape* shape, const rf_params* params, RfGeom* out);
 
 struct RfAttnArgs {
   RfGeom g;

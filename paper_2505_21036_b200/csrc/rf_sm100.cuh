@@ -24,16 +24,22 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+// Potentially-blocking test: the hardware may suspend the thread for a bounded time before answering.
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
       : "memory");
   return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
 }
 
 struct WaitCtx {
@@ -41,15 +47,15 @@ struct WaitCtx {
   int32_t* dev_status;       // global, may be null
 };
 
-// Bounded wait (about a second at most).  Returns false if the wait was abandoned.
+// Bounded wait: two seconds of wall clock (and an iteration cap) at most.  Returns false if the wait
+// was abandoned; from then on every wait of the CTA returns at once.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
-  constexpr uint32_t kSpin = 1u << 14, kLimit = 1u << 22;
-  for (uint32_t it = 0; it < kLimit; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if (it >= kSpin) {
-      if (*w.abort_flag) return false;
-      __nanosleep(128);
-    }
+  if (mbar_try(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t it = 0; it < (1u << 26); ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if (*w.abort_flag) return false;
+    if (global_timer_ns() - t0 > 2000000000ull) break;
   }
   *w.abort_flag = 1;
   rf_report(w.dev_status, RF_ERR_TIMEOUT);

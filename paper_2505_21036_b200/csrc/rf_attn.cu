@@ -334,72 +334,78 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       const int u0 = (int)(entry & ~RF_PARTIAL_BIT) * BN;
       mbar_wait(bar(C::B_SF + j), it & 1, wc);
       tc_fence_after();
-      uint32_t s[128];
-      {
-        uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
-        uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
-        uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
-        uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
-        tmem_ld32(t_s, s0);
-        tmem_ld32(t_s + 32, s1);
-        tmem_ld32(t_s + 64, s2);
-        tmem_ld32(t_s + 96, s3);
-        tc_wait_ld();
-      }
-      if (partial) {
-        uint32_t w[4];
-        rmask.tile_bits(u0, w);
-#pragma unroll
-        for (int c = 0; c < 128; ++c)
-          if (!((w[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 128; c += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(s[c]));
-        mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
-        mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
-      }
-      const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc;
-
-      // raise the running maximum only when it grows by more than the threshold
-      const bool raise = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
-      float alpha = 1.f;
-      if (raise) {
-        alpha = ex2(m_run - m_tile);   // 0 when m_run = -inf
-        m_run = m_tile;
-        l_run *= alpha;
-      }
-      if (it > 0 && __any_sync(0xffffffffu, raise)) {
-        // O of the previous tiles must be complete before it is rescaled
-        mbar_wait(bar(C::B_OF + j), (it - 1) & 1, wc);
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(t_o + c * 32, v);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-          tmem_st32(t_o + c * 32, v);
-        }
-        tc_wait_st();
-      }
-      const float m_use = m_run == -INFINITY ? 0.f : m_run;
-      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+      // Exponentials are taken against the running maximum of the previous tiles while the tile's own
+      // maximum is computed alongside; only if some row's maximum grew by more than the threshold
+      // (rare after the first tile) is the running maximum raised, O rescaled and the pass repeated
+      // (S is still in TMEM then: P has not been stored yet).
       uint32_t pk[64];
+#pragma unroll 1
+      for (int pass = 0; pass < 2; ++pass) {
+        uint32_t s[128];
+        {
+          uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+          uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+          uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+          uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+          tmem_ld32(t_s, s0);
+          tmem_ld32(t_s + 32, s1);
+          tmem_ld32(t_s + 64, s2);
+          tmem_ld32(t_s + 96, s3);
+          tc_wait_ld();
+        }
+        if (partial) {
+          uint32_t w[4];
+          rmask.tile_bits(u0, w);
 #pragma unroll
-      for (int c = 0; c < 128; c += 4) {
-        const float p0 = ex2(fmaf(__uint_as_float(s[c]), sc, -m_use));
-        const float p1 = ex2(fmaf(__uint_as_float(s[c + 1]), sc, -m_use));
-        const float p2 = ex2(fmaf(__uint_as_float(s[c + 2]), sc, -m_use));
-        const float p3 = ex2(fmaf(__uint_as_float(s[c + 3]), sc, -m_use));
-        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-        pk[c / 2] = pack_bf16(p0, p1);
-        pk[c / 2 + 1] = pack_bf16(p2, p3);
+          for (int c = 0; c < 128; ++c)
+            if (!((w[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf
+        }
+        const float m_use = m_run == -INFINITY ? 0.f : m_run;
+        const float2 sc2 = make_float2(sc, sc), mneg = make_float2(-m_use, -m_use);
+        float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 128; c += 4) {
+          const float s0 = __uint_as_float(s[c]), s1 = __uint_as_float(s[c + 1]);
+          const float s2 = __uint_as_float(s[c + 2]), s3 = __uint_as_float(s[c + 3]);
+          mx0 = fmaxf(mx0, fmaxf(s0, s1));
+          mx1 = fmaxf(mx1, fmaxf(s2, s3));
+          float2 e0 = __ffma2_rn(make_float2(s0, s1), sc2, mneg);
+          float2 e1 = __ffma2_rn(make_float2(s2, s3), sc2, mneg);
+          e0.x = ex2(e0.x); e0.y = ex2(e0.y);
+          e1.x = ex2(e1.x); e1.y = ex2(e1.y);
+          la = __fadd2_rn(la, e0);
+          lb = __fadd2_rn(lb, e1);
+          pk[c / 2] = pack_bf16(e0.x, e0.y);
+          pk[c / 2 + 1] = pack_bf16(e1.x, e1.y);
+        }
+        const float l_tile = (la.x + la.y) + (lb.x + lb.y);
+        if (pass == 1) { l_run += l_tile; break; }
+        const float m_tile = fmaxf(mx0, mx1) * sc;
+        const bool raise = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
+        if (!__any_sync(0xffffffffu, raise)) { l_run += l_tile; break; }
+        float alpha = 1.f;
+        if (raise) {
+          alpha = ex2(m_run - m_tile);   // 0 when m_run = -inf
+          m_run = m_tile;
+          l_run *= alpha;
+        }
+        if (it > 0) {
+          // O of the previous tiles must be complete before it is rescaled
+          mbar_wait(bar(C::B_OF + j), (it - 1) & 1, wc);
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(t_o + c * 32, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+            tmem_st32(t_o + c * 32, v);
+          }
+          tc_wait_st();
+        }
       }
-      l_run += (l0 + l1) + (l2 + l3);
       {
         uint32_t(&p0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[0]);
         uint32_t(&p1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[32]);

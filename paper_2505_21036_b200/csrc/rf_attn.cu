@@ -253,24 +253,30 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
+      // Descriptors differ only in their 14-bit start-address field: keep the constant words in
+      // registers and add the byte offset (>> 4) per k-step.
+      constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);      // SBO 1024 B, version 1, 128B swizzle
+      constexpr uint32_t LO_KMAJOR = 1u << 16;                                    // LBO field unused for K-major
+      constexpr uint32_t LO_VMAJOR = (C::BLK >> 4) << 16;                         // LBO = one 64-column block
+      auto desc = [](uint32_t lo) -> uint64_t { return ((uint64_t)DESC_HI << 32) | lo; };
+      const uint32_t q_lo = ((base + C::Q) >> 4) | LO_KMAJOR, k_lo = ((base + C::K0) >> 4) | LO_KMAJOR;
+      const uint32_t v_lo = ((base + C::V0) >> 4) | LO_VMAJOR;
       auto issue_s = [&](int j, int ks) {
+        const uint32_t a0 = q_lo + j * (C::TILE >> 4), b0 = k_lo + ks * (C::TILE >> 4);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t off = C::koff(k);
-          mma_ss(tmem_base + (j ? C::S_COL1 : C::S_COL0), smem_desc_sw128(base + C::Q + j * C::TILE + off, 16, 1024),
-                 smem_desc_sw128(base + C::K0 + ks * C::TILE + off, 16, 1024), IDESC_S, k > 0);
-        }
+        for (int k = 0; k < D / 16; ++k)
+          mma_ss(tmem_base + (j ? C::S_COL1 : C::S_COL0), desc(a0 + (C::koff(k) >> 4)), desc(b0 + (C::koff(k) >> 4)),
+                 IDESC_S, k > 0);
         tc_commit(bar(C::B_SF + j));
       };
       auto issue_pv = [&](int j, int vs, bool first) {
+        const uint32_t b0 = v_lo + vs * (C::TILE >> 4);
+        const uint32_t t_p = tmem_base + (j ? C::S_COL1 : C::S_COL0), t_o = tmem_base + (j ? C::O_COL1 : C::O_COL0);
 #pragma unroll
         for (int k = 0; k < BN / 16; ++k) {
-          mma_ts(tmem_base + (j ? C::O_COL1 : C::O_COL0), tmem_base + (j ? C::S_COL1 : C::S_COL0) + k * 8,
-                 smem_desc_sw128(base + C::V0 + vs * C::TILE + k * 2048, C::BLK, 1024), IDESC_PV, (!first) || k > 0);
+          mma_ts(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
           if (D == 96)  // columns [64, 96): the upper half of the second block's 128-byte rows
-            mma_ts(tmem_base + (j ? C::O_COL1 : C::O_COL0) + 64, tmem_base + (j ? C::S_COL1 : C::S_COL0) + k * 8,
-                   smem_desc_sw128(base + C::V0 + vs * C::TILE + C::BLK + k * 2048 + 64, C::BLK, 1024), IDESC_PV32,
-                   (!first) || k > 0);
+            mma_ts(t_o + 64, t_p + k * 8, desc(b0 + ((C::BLK + k * 2048 + 64) >> 4)), IDESC_PV32, (!first) || k > 0);
         }
         tc_commit(bar(C::B_OF + j));
       };

@@ -35,7 +35,7 @@ struct Cfg {
   static constexpr uint32_t BLK = 128 * 128;          // bytes of one 128-row x 64-col bf16 block
   static constexpr uint32_t TILE = KB * BLK;          // bytes of one 128-row tile
   static constexpr int NK = D == 64 ? 4 : 2;          // K ring depth
-  static constexpr int NV = D == 64 ? 4 : 2;          // V ring depth
+  static constexpr int NV = D == 64 ? 4 : 3;          // V ring depth
   // byte offset, inside a tile, of the 16 columns of k-step ks of the Q K^T contraction
   static __host__ __device__ constexpr uint32_t koff(int ks) {
     return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks * 16 - COL1) * 2u;
@@ -139,15 +139,18 @@ struct Lists {
 };
 struct Merge {
   int i0 = 0, i1 = 0;
+  int h0, h1;   // heads of the two lists, loaded one call ahead so that their latency is off the critical path
+  __device__ __forceinline__ void start(const Lists& L) {
+    h0 = L.n0 > 0 ? (int)(L.entry(0, 0) & ~RF_PARTIAL_BIT) : 0x7fffffff;
+    h1 = L.n1 > 0 ? (int)(L.entry(1, 0) & ~RF_PARTIAL_BIT) : 0x7fffffff;
+  }
   // Next tile of the union; uses bit j set when stream j lists it.  Returns false when exhausted.
   __device__ __forceinline__ bool next(const Lists& L, int& tile, int& uses) {
-    const int e0 = i0 < L.n0 ? (int)(L.entry(0, i0) & ~RF_PARTIAL_BIT) : 0x7fffffff;
-    const int e1 = i1 < L.n1 ? (int)(L.entry(1, i1) & ~RF_PARTIAL_BIT) : 0x7fffffff;
-    tile = min(e0, e1);
+    tile = min(h0, h1);
     if (tile == 0x7fffffff) return false;
-    uses = (e0 == tile ? 1 : 0) | (e1 == tile ? 2 : 0);
-    i0 += e0 == tile;
-    i1 += e1 == tile;
+    uses = (h0 == tile ? 1 : 0) | (h1 == tile ? 2 : 0);
+    if (uses & 1) { ++i0; h0 = i0 < L.n0 ? (int)(L.entry(0, i0) & ~RF_PARTIAL_BIT) : 0x7fffffff; }
+    if (uses & 2) { ++i1; h1 = i1 < L.n1 ? (int)(L.entry(1, i1) & ~RF_PARTIAL_BIT) : 0x7fffffff; }
     return true;
   }
 };
@@ -235,6 +238,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         for (int kb = 0; kb < KB; ++kb)
           tma_load_3d(base + C::Q + j * C::TILE + kb * C::BLK, map_q, kb * C::COL1, (qt0 + j) * BM, bh, bar(C::B_Q));
       Merge mg;
+      mg.start(L);
       int tile, uses;
       for (int u = 0; mg.next(L, tile, uses); ++u) {
         const int ks = u % C::NK, vs = u % C::NV;
@@ -281,6 +285,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         tc_commit(bar(C::B_OF + j));
       };
       Merge mg;
+      mg.start(L);
       int cur_tile, cur_uses, nxt_tile = 0, nxt_uses = 0;
       bool has_cur = mg.next(L, cur_tile, cur_uses);
       int pv_cnt[2] = {0, 0};

@@ -1,19 +1,27 @@
 // ARM: Adaptive Recognition Module (Sec. 3.3, Eq. 6, Algorithm 1).
 //
-// For a sample I of video tokens (the first frame, or every omega-th token) each CTA takes 64
-// sampled query rows and streams all sampled keys through shared memory in blocks of 64:
-// scores on the tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate), online softmax in fp32
-// with warp shuffles for the row maximum, and next to the total mass three masked masses: the
-// part of the row kept by the Temporal, the Spatial and the Textural mask restricted to I.
+// For a sample I of video tokens (the first frame, or every omega-th token) each CTA takes 128
+// sampled query rows and streams all sampled keys through shared memory in blocks of 64 (cp.async,
+// double-buffered): scores on the tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate), online
+// softmax in fp32 with warp shuffles for the row maximum, and next to the total mass the masked
+// masses: the part of the row kept by the Temporal, the Spatial and (when recalls are wanted) the
+// Textural mask restricted to I.  A key block that lies wholly inside or outside a mask's band for
+// all 16 rows of a warp is settled per block (frames grow monotonically with the sample index, and
+// on the first-frame sample so do positions); only blocks a band edge crosses test per element.
 // The n x n score matrix is never written.  Per-row recalls go to scratch; a second kernel
 // averages them in a fixed order (deterministic) and takes Algorithm 1's decision.
 #include "rf_common.cuh"
 
 namespace {
 
-constexpr int ARM_ROWS = 64;   // query rows per CTA (16 per warp)
+constexpr int ARM_ROWS = 128;  // query rows per CTA (16 per warp)
 constexpr int ARM_KEYS = 64;   // keys per shared-memory block
-constexpr int ARM_THREADS = 128;
+constexpr int ARM_THREADS = 256;
+
+// Which masked masses a launch accumulates.
+constexpr int ARM_LOCAL_T = 0;    // first-frame sample: Temporal only (positions = sample index)
+constexpr int ARM_GLOBAL_S = 1;   // stride sample: Spatial
+constexpr int ARM_GLOBAL_ST = 2;  // stride sample: Spatial and Temporal
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -28,6 +36,21 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// 16-byte asynchronous copy; zero-fills when !valid (src must still be a readable address).
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 struct KeyAttr { int f, p, c; };  // frame, in-frame position, 1 if in the checkerboard set C
 
 __device__ __forceinline__ KeyAttr token_attr(const RfGeom& g, int tok) {
@@ -39,71 +62,91 @@ __device__ __forceinline__ KeyAttr token_attr(const RfGeom& g, int tok) {
   return a;
 }
 
-// grid = (ceil(n/64), B*H).  stride: token index of sample m is m*stride.
-// row_out: [B*H][3][n_pad] per-row recalls (temporal, spatial, textural) of this sample.
-template <int D>
+// 0: no pair of (rows, cols) within w, 2: every pair within w, 1: mixed.  Closed integer ranges.
+__device__ __forceinline__ int band_class(int ra, int rb, int ca, int cb, int w) {
+  const int dmin = max(max(ca - rb, ra - cb), 0), dmax = max(rb - ca, cb - ra);
+  return dmax <= w ? 2 : (dmin > w ? 0 : 1);
+}
+
+// grid = (ceil(n/128), B*H).  stride: token index of sample m is m*stride.
+// row_out: [B*H][3][n_pad] per-row recalls (temporal, spatial, textural) of this sample; only the
+// masses this launch accumulates are written.
+template <int D, int MODE, bool TEX>
 __global__ void __launch_bounds__(ARM_THREADS) rf_arm_rows_kernel(RfGeom g, int n, int stride, int n_pad,
                                                                    const __nv_bfloat16* __restrict__ q,
                                                                    const __nv_bfloat16* __restrict__ k,
                                                                    float scale_log2, float* __restrict__ row_out) {
   constexpr int LD = D + 8;  // padded row, keeps ldmatrix conflict-free
-  __shared__ __align__(16) __nv_bfloat16 Qs[ARM_ROWS * LD];
-  __shared__ __align__(16) __nv_bfloat16 Ks[ARM_KEYS * LD];
-  __shared__ int kf[ARM_KEYS], kp[ARM_KEYS], kc[ARM_KEYS];
+  constexpr int VEC = D / 8;
+  constexpr bool WANT_T = MODE != ARM_GLOBAL_S, WANT_S = MODE != ARM_LOCAL_T;
+  constexpr bool T_BAND = MODE == ARM_LOCAL_T;  // Temporal mask is a band in sample-index space
+  // the Q tile first; once its fragments are in registers the same memory holds two key blocks
+  __shared__ __align__(16) __nv_bfloat16 buf[ARM_ROWS * LD];
+  __shared__ int kf[2][ARM_KEYS], kp[2][ARM_KEYS], kc[2][ARM_KEYS];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int bh = blockIdx.y;
   const int row0 = blockIdx.x * ARM_ROWS;
   const size_t head = (size_t)bh * g.N * D;
-  constexpr int VEC = D / 8;
 
   for (int i = tid; i < ARM_ROWS * VEC; i += ARM_THREADS) {
     const int r = i / VEC, c = i % VEC;
-    const int m = row0 + r;
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if (m < n) val = __ldg(reinterpret_cast<const uint4*>(q + head + (size_t)m * stride * D) + c);
-    *reinterpret_cast<uint4*>(&Qs[r * LD + c * 8]) = val;
+    const int m = min(row0 + r, n - 1);
+    cp_async16(smem_u32(&buf[r * LD + c * 8]), q + head + (size_t)m * stride * D + c * 8, true);
   }
+  cp_async_commit();
+  cp_async_wait<0>();
   __syncthreads();
 
   uint32_t qa[D / 16][4];
 #pragma unroll
   for (int ks = 0; ks < D / 16; ++ks) {
-    const uint32_t addr = smem_u32(&Qs[(warp * 16 + (lane & 15)) * LD + ks * 16 + (lane >> 4) * 8]);
+    const uint32_t addr = smem_u32(&buf[(warp * 16 + (lane & 15)) * LD + ks * 16 + (lane >> 4) * 8]);
     ldmatrix_x4(addr, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
   }
+  __syncthreads();  // every warp has its fragments: the buffer may be overwritten with keys
+
+  auto load_keys = [&](int blk) {
+    const int k0 = blk * ARM_KEYS, b = blk & 1;
+    for (int i = tid; i < ARM_KEYS * VEC; i += ARM_THREADS) {
+      const int r = i / VEC, c = i % VEC;
+      const int m = k0 + r;
+      cp_async16(smem_u32(&buf[(b * ARM_KEYS + r) * LD + c * 8]), k + head + (size_t)min(m, n - 1) * stride * D + c * 8, m < n);
+    }
+    if (tid < ARM_KEYS) {
+      const KeyAttr a = token_attr(g, min(k0 + tid, n - 1) * stride);
+      kf[b][tid] = a.f; kp[b][tid] = a.p; kc[b][tid] = a.c;
+    }
+    cp_async_commit();
+  };
 
   // the two rows this thread sees: warp*16 + lane/4 and +8
   int rf[2], rp[2];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    const int m = min(row0 + warp * 16 + (lane >> 2) + h * 8, n - 1);
-    const KeyAttr a = token_attr(g, m * stride);
+    const KeyAttr a = token_attr(g, min(row0 + warp * 16 + (lane >> 2) + h * 8, n - 1) * stride);
     rf[h] = a.f;
     rp[h] = a.p;
   }
+  // row range of this warp, for the per-block band classification
+  const int wra = min(row0 + warp * 16, n - 1), wrb = min(row0 + warp * 16 + 15, n - 1);
+  const int wfa = (wra * stride) / g.S, wfb = (wrb * stride) / g.S;
+
   float mx[2] = {-INFINITY, -INFINITY};
   float l_all[2] = {0.f, 0.f}, l_t[2] = {0.f, 0.f}, l_s[2] = {0.f, 0.f}, l_c[2] = {0.f, 0.f};
 
-  for (int k0 = 0; k0 < n; k0 += ARM_KEYS) {
-    __syncthreads();  // previous block fully consumed
-    for (int i = tid; i < ARM_KEYS * VEC; i += ARM_THREADS) {
-      const int r = i / VEC, c = i % VEC;
-      const int m = k0 + r;
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (m < n) val = __ldg(reinterpret_cast<const uint4*>(k + head + (size_t)m * stride * D) + c);
-      *reinterpret_cast<uint4*>(&Ks[r * LD + c * 8]) = val;
-    }
-    if (tid < ARM_KEYS) {
-      const int m = k0 + tid;
-      if (m < n) {
-        const KeyAttr a = token_attr(g, m * stride);
-        kf[tid] = a.f; kp[tid] = a.p; kc[tid] = a.c;
-      } else {
-        kf[tid] = -1; kp[tid] = 0; kc[tid] = 0;  // f = -1 marks a slot past the sample
-      }
+  const int nblk = rf_cdiv(n, ARM_KEYS);
+  load_keys(0);
+  for (int blk = 0; blk < nblk; ++blk) {
+    const int k0 = blk * ARM_KEYS, b = blk & 1;
+    if (blk + 1 < nblk) {
+      load_keys(blk + 1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
     }
     __syncthreads();
+    const __nv_bfloat16* Ks = buf + b * ARM_KEYS * LD;
 
     float acc[ARM_KEYS / 8][4];
 #pragma unroll
@@ -121,40 +164,59 @@ __global__ void __launch_bounds__(ARM_THREADS) rf_arm_rows_kernel(RfGeom g, int 
       }
     }
 
-    // scale to the log2 domain, mask slots past the sample, block row maximum
+    // key slots past the sample (last block only) carry -inf
+    if (k0 + ARM_KEYS > n) {
+#pragma unroll
+      for (int nt = 0; nt < ARM_KEYS / 8; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (k0 + nt * 8 + (lane & 3) * 2 + (e & 1) >= n) acc[nt][e] = -INFINITY;
+    }
     float bm[2] = {-INFINITY, -INFINITY};
 #pragma unroll
     for (int nt = 0; nt < ARM_KEYS / 8; ++nt) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
-        const float s = kf[col] < 0 ? -INFINITY : acc[nt][e] * scale_log2;
-        acc[nt][e] = s;
-        bm[e >> 1] = fmaxf(bm[e >> 1], s);
-      }
+      bm[0] = fmaxf(bm[0], fmaxf(acc[nt][0], acc[nt][1]));
+      bm[1] = fmaxf(bm[1], fmaxf(acc[nt][2], acc[nt][3]));
     }
+    float neg_m[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       bm[h] = fmaxf(bm[h], __shfl_xor_sync(0xffffffffu, bm[h], 1));
       bm[h] = fmaxf(bm[h], __shfl_xor_sync(0xffffffffu, bm[h], 2));
-      const float m_new = fmaxf(mx[h], bm[h]);           // finite: every block holds >= 1 real key
-      const float corr = exp2f(mx[h] - m_new);           // exp2(-inf) = 0 on the first block
+      const float m_new = fmaxf(mx[h], bm[h] * scale_log2);   // finite: every block holds >= 1 real key
+      const float corr = ex2f(mx[h] - m_new);                  // 0 on the first block
       l_all[h] *= corr; l_t[h] *= corr; l_s[h] *= corr; l_c[h] *= corr;
       mx[h] = m_new;
+      neg_m[h] = -m_new;
     }
+
+    // band classes of this block for the warp's 16 rows (warp-uniform)
+    const int ca = k0, cb = min(k0 + ARM_KEYS - 1, n - 1);
+    const int t_cls = !WANT_T ? 0 : (T_BAND ? band_class(wra, wrb, ca, cb, g.ws) : 1);
+    const int s_cls = !WANT_S ? 0 : band_class(wfa, wfb, (ca * stride) / g.S, (cb * stride) / g.S, g.wf);
+
+    float bs[2] = {0.f, 0.f}, bt[2] = {0.f, 0.f}, bsp[2] = {0.f, 0.f}, bc[2] = {0.f, 0.f};
 #pragma unroll
     for (int nt = 0; nt < ARM_KEYS / 8; ++nt) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int h = e >> 1;
         const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
-        const float p = exp2f(acc[nt][e] - mx[h]);
-        l_all[h] += p;
-        if (abs(kp[col] - rp[h]) <= g.ws) l_t[h] += p;
-        if (abs(kf[col] - rf[h]) <= g.wf) l_s[h] += p;
-        if (kc[col]) l_c[h] += p;
+        const float p = ex2f(fmaf(acc[nt][e], scale_log2, neg_m[h]));
+        bs[h] += p;
+        if (WANT_T && t_cls == 1) { if (abs(kp[b][col] - rp[h]) <= g.ws) bt[h] += p; }
+        if (WANT_S && s_cls == 1) { if (abs(kf[b][col] - rf[h]) <= g.wf) bsp[h] += p; }
+        if (TEX) { if (kc[b][col]) bc[h] += p; }
       }
     }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      l_all[h] += bs[h];
+      if (WANT_T) l_t[h] += t_cls == 2 ? bs[h] : bt[h];
+      if (WANT_S) l_s[h] += s_cls == 2 ? bs[h] : bsp[h];
+      if (TEX) l_c[h] += bc[h];
+    }
+    __syncthreads();  // block consumed: its buffer is the target of the next prefetch
   }
 
   // quad reduction of the partial masses, then one lane per row writes its recalls
@@ -171,9 +233,9 @@ __global__ void __launch_bounds__(ARM_THREADS) rf_arm_rows_kernel(RfGeom g, int 
     if ((lane & 3) == 0 && m < n) {
       float* out = row_out + (size_t)bh * 3 * n_pad;
       const float inv = 1.f / l_all[h];
-      out[m] = l_t[h] * inv;
-      out[n_pad + m] = l_s[h] * inv;
-      out[2 * n_pad + m] = l_c[h] * inv;
+      if (WANT_T) out[m] = l_t[h] * inv;
+      if (WANT_S) out[n_pad + m] = l_s[h] * inv;
+      if (TEX) out[2 * n_pad + m] = l_c[h] * inv;
     }
   }
 }
@@ -190,9 +252,11 @@ __global__ void __launch_bounds__(256) rf_arm_decide_kernel(int n_loc, int n_glb
   const bool local_t = sample_mode == RF_SAMPLE_ALG1;
   const float* src[3] = {local_t ? lo : gl, gl + n_pad, gl + 2 * n_pad};
   const int cnt[3] = {local_t ? n_loc : n_glb, n_glb, n_glb};
+  const int nw = recall != nullptr ? 3 : 2;   // the Textural recall is only accumulated when recalls are wanted
   for (int w = 0; w < 3; ++w) {
     double s = 0.0;
-    for (int i = tid; i < cnt[w]; i += 256) s += (double)src[w][i];
+    if (w < nw)
+      for (int i = tid; i < cnt[w]; i += 256) s += (double)src[w][i];
     red[w][tid] = s;
   }
   __syncthreads();
@@ -208,21 +272,32 @@ __global__ void __launch_bounds__(256) rf_arm_decide_kernel(int n_loc, int n_glb
   }
 }
 
-template <int D>
+template <int D, int MODE, bool TEX>
 cudaError_t launch_rows(const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q, const __nv_bfloat16* k,
                         float* out, cudaStream_t st) {
   dim3 grid(rf_cdiv(n, ARM_ROWS), g.B * g.H);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
-  rf_arm_rows_kernel<D><<<grid, ARM_THREADS, 0, st>>>(g, n, stride, n_pad, q, k, scale_log2, out);
+  rf_arm_rows_kernel<D, MODE, TEX><<<grid, ARM_THREADS, 0, st>>>(g, n, stride, n_pad, q, k, scale_log2, out);
   return cudaGetLastError();
 }
 
-cudaError_t launch_rows_d(const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q, const __nv_bfloat16* k,
-                          float* out, cudaStream_t st) {
+template <int D>
+cudaError_t launch_rows_m(int mode, bool tex, const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q,
+                          const __nv_bfloat16* k, float* out, cudaStream_t st) {
+  if (mode == ARM_LOCAL_T) return launch_rows<D, ARM_LOCAL_T, false>(g, n, stride, n_pad, q, k, out, st);
+  if (mode == ARM_GLOBAL_S)
+    return tex ? launch_rows<D, ARM_GLOBAL_S, true>(g, n, stride, n_pad, q, k, out, st)
+               : launch_rows<D, ARM_GLOBAL_S, false>(g, n, stride, n_pad, q, k, out, st);
+  return tex ? launch_rows<D, ARM_GLOBAL_ST, true>(g, n, stride, n_pad, q, k, out, st)
+             : launch_rows<D, ARM_GLOBAL_ST, false>(g, n, stride, n_pad, q, k, out, st);
+}
+
+cudaError_t launch_rows_d(int mode, bool tex, const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q,
+                          const __nv_bfloat16* k, float* out, cudaStream_t st) {
   switch (g.D) {
-    case 64: return launch_rows<64>(g, n, stride, n_pad, q, k, out, st);
-    case 96: return launch_rows<96>(g, n, stride, n_pad, q, k, out, st);
-    case 128: return launch_rows<128>(g, n, stride, n_pad, q, k, out, st);
+    case 64: return launch_rows_m<64>(mode, tex, g, n, stride, n_pad, q, k, out, st);
+    case 96: return launch_rows_m<96>(mode, tex, g, n, stride, n_pad, q, k, out, st);
+    case 128: return launch_rows_m<128>(mode, tex, g, n, stride, n_pad, q, k, out, st);
   }
   return cudaErrorInvalidValue;
 }
@@ -244,10 +319,12 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
   const int n_glb = rf_cdiv(g.Nv, omega), n_loc = g.S;
   float* rows_glb = row_scratch;
   float* rows_loc = row_scratch + (size_t)g.B * g.H * 3 * n_pad;
-  cudaError_t e = launch_rows_d(g, n_glb, omega, n_pad, q, k, rows_glb, st);
+  const bool alg1 = sample_mode == RF_SAMPLE_ALG1;
+  const bool tex = recall != nullptr;   // the Textural recall is a diagnostic: Algorithm 1 does not use it
+  cudaError_t e = launch_rows_d(alg1 ? ARM_GLOBAL_S : ARM_GLOBAL_ST, tex, g, n_glb, omega, n_pad, q, k, rows_glb, st);
   if (e != cudaSuccess) return e;
-  if (sample_mode == RF_SAMPLE_ALG1) {
-    e = launch_rows_d(g, n_loc, 1, n_pad, q, k, rows_loc, st);
+  if (alg1) {
+    e = launch_rows_d(ARM_LOCAL_T, false, g, n_loc, 1, n_pad, q, k, rows_loc, st);
     if (e != cudaSuccess) return e;
   }
   rf_arm_decide_kernel<<<g.B * g.H, 256, 0, st>>>(n_loc, n_glb, n_pad, sample_mode, alpha, rows_loc, rows_glb,

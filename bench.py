@@ -149,19 +149,15 @@ def run_reference(args, wl):
 
 def run_cuda(args, wl):
     import torch
-    import torch.distributed as dist
-    from paper_2505_21036_b200 import api
+    from paper_2505_21036_b200 import api, dist_util
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
     api.load()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = dist_util.env_rank()
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
+    dist_util.init("nccl", dev)
 
     # inputs: seeded on the host (pinned, for the end-to-end leg), resident copy on the device
     qh, kh, vh = (torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in synth.make_qkv(wl))
@@ -194,8 +190,7 @@ def run_cuda(args, wl):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        dist_util.barrier()
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -260,10 +255,7 @@ def run_cuda(args, wl):
         raise SystemExit(f"bench.py: device status {int(status.item())}")
 
     ms_per_step = total_ms / args.steps
-    t = torch.tensor([ms_per_step, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step, e2e_ms = dist_util.max_over_ranks([ms_per_step, e2e_ms], dev)
 
     if rank == 0:
         pk = peaks()
@@ -272,7 +264,7 @@ def run_cuda(args, wl):
         attn_kernel_ms = max(sparse_ms - reorder_ms, 1e-6)
         achieved = tile_flops / (attn_kernel_ms * 1e-3) / 1e12
         line = {
-            "metric": METRIC, "value": world * dflops / (ms_per_step * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": dist_util.replica_throughput(dflops, ms_per_step, world) / 1e12, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "D": wl.D, "T": wl.T, "frame": [wl.frame_h, wl.frame_w],
@@ -281,7 +273,7 @@ def run_cuda(args, wl):
                        "textural_stride": wl.textural_stride, "sample_stride": wl.sample_stride,
                        "l2": "inputs (2.2 GB of Q/K/V) exceed L2", "parallelism": f"replicas x{world}"},
             "clocks": clocks,
-            "e2e": {"value": world * dflops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": dist_util.replica_throughput(dflops, e2e_ms, world) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": o.numel() * 2},
             "gpu_launches": args.steps * (6 if wl.sample_mode == 0 else 5),
             "breakdown_ms": {"arm": arm_ms, "block_mask": mask_ms, "sparse_attn_call": sparse_ms, "reorder": reorder_ms,
@@ -306,8 +298,7 @@ def run_cuda(args, wl):
                                     "sample": f"head 0: ARM + masked attention on {nrows} of {wl.N} query rows, "
                                               f"{dt:.1f} s, extrapolated by rows"}
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    dist_util.shutdown()
 
 
 def main():

@@ -1,0 +1,87 @@
+"""Host side of the C ABI without a GPU: the library builds, loads, exports every function the header
+declares, and rejects bad arguments before anything touches CUDA."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2505_21036_b200 import api, build, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return api.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "rainfusion.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rf_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_function_is_exported(lib):
+    names = declared_functions()
+    assert {"rf_arm_classify", "rf_build_block_mask", "rf_sparse_attn_fwd", "rf_dense_attn_fwd"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(api.EXPORTS) <= set(names)
+
+
+def test_status_strings(lib):
+    assert lib.rf_status_string(0) == b"ok"
+    for code in range(1, 7):
+        assert lib.rf_status_string(code) not in (b"ok", b"unknown status")
+    assert lib.rf_status_string(99) == b"unknown status"
+
+
+def test_schedule_dims_and_workspace_for_every_workload(lib):
+    for wl in synth.WORKLOADS.values():
+        s, p = api.shape_of(wl), api.params_of(wl)
+        nq, nk = api.rf_schedule_dims(s, p)
+        assert nq == nk == -(-wl.N // 128)
+        tensor = -(-(wl.B * wl.H * wl.N * wl.D * 2) // 256) * 256
+        assert api.rf_workspace_bytes(s, p) >= 3 * tensor
+    wl = synth.WORKLOADS["tiny"]
+    assert api.rf_schedule_dims(api.shape_of(wl), api.params_of(wl, 16, 32)) == (17, 9)
+
+
+@pytest.mark.parametrize("field,value", [("frame_window", -1), ("spatial_window", -1), ("textural_stride", 0),
+                                         ("sample_stride", 0), ("sample_mode", 2), ("alpha", 0.0), ("alpha", 1.5),
+                                         ("block_m", 48), ("block_n", 8), ("temporal_permute", 2)])
+def test_bad_parameters_are_rejected(lib, field, value):
+    wl = synth.WORKLOADS["tiny"]
+    s, p = api.shape_of(wl), api.params_of(wl)
+    setattr(p, field, value)
+    assert lib.rf_schedule_dims(C.byref(s), C.byref(p), None, None) == 1
+    assert lib.rf_workspace_bytes(C.byref(s), C.byref(p)) == 0
+
+
+def test_bad_shapes_and_pointers_are_rejected_before_cuda(lib):
+    wl = synth.WORKLOADS["tiny"]
+    s, p = api.shape_of(wl), api.params_of(wl)
+    bad = api.make_shape(1, 3, 64, 0, 8, 8, 16)
+    assert lib.rf_schedule_dims(C.byref(bad), C.byref(p), None, None) == 1
+    odd = api.make_shape(1, 3, 80, 4, 8, 8, 16)                       # head dimension not supported by attention
+    assert lib.rf_dense_attn_fwd(C.byref(odd), 256, 256, 256, 256, None, None, 0, None, None) == 2
+    # null and misaligned pointers
+    assert lib.rf_dense_attn_fwd(C.byref(s), None, 256, 256, 256, None, None, 0, None, None) == 1
+    assert lib.rf_dense_attn_fwd(C.byref(s), 264, 256, 256, 256, None, None, 0, None, None) == 1
+    assert lib.rf_arm_classify(C.byref(s), C.byref(p), 256, 256, None, None, 256, 1 << 30, None) == 1
+    assert lib.rf_arm_classify(C.byref(s), C.byref(p), 256, 256, 256, None, 256, 16, None) == 3   # workspace too small
+    sched = api.rf_schedule(256, 256, None, 256, 1, 1)                # wrong nQ / nKmax
+    assert lib.rf_build_block_mask(C.byref(s), C.byref(p), 256, C.byref(sched), None, None) == 1
+    p64 = api.params_of(wl, 64, 64)
+    sched = api.rf_schedule(256, 256, None, 256, 5, 5)
+    assert lib.rf_sparse_attn_fwd(C.byref(s), C.byref(p64), 256, 256, 256, 256, C.byref(sched), 256, None, 256,
+                                  1 << 30, None, None) == 2            # attention needs 128 x 128 tiles
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(api, "_lib", None)
+    monkeypatch.setattr(api, "_LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(api.RainFusionError):
+        api.load()

@@ -139,18 +139,22 @@ struct Lists {
 };
 struct Merge {
   int i0 = 0, i1 = 0;
-  int h0, h1;   // heads of the two lists, loaded one call ahead so that their latency is off the critical path
+  // Raw list entries at i0 / i1, loaded by the previous call and not touched until the next one, so
+  // that the load latency never sits between two MMA bursts of the (in-order) issuing thread.
+  uint32_t raw0 = 0, raw1 = 0;
   __device__ __forceinline__ void start(const Lists& L) {
-    h0 = L.n0 > 0 ? (int)(L.entry(0, 0) & ~RF_PARTIAL_BIT) : 0x7fffffff;
-    h1 = L.n1 > 0 ? (int)(L.entry(1, 0) & ~RF_PARTIAL_BIT) : 0x7fffffff;
+    if (L.n0 > 0) raw0 = L.entry(0, 0);
+    if (L.n1 > 0) raw1 = L.entry(1, 0);
   }
   // Next tile of the union; uses bit j set when stream j lists it.  Returns false when exhausted.
   __device__ __forceinline__ bool next(const Lists& L, int& tile, int& uses) {
+    const int h0 = i0 < L.n0 ? (int)(raw0 & ~RF_PARTIAL_BIT) : 0x7fffffff;
+    const int h1 = i1 < L.n1 ? (int)(raw1 & ~RF_PARTIAL_BIT) : 0x7fffffff;
     tile = min(h0, h1);
     if (tile == 0x7fffffff) return false;
     uses = (h0 == tile ? 1 : 0) | (h1 == tile ? 2 : 0);
-    if (uses & 1) { ++i0; h0 = i0 < L.n0 ? (int)(L.entry(0, i0) & ~RF_PARTIAL_BIT) : 0x7fffffff; }
-    if (uses & 2) { ++i1; h1 = i1 < L.n1 ? (int)(L.entry(1, i1) & ~RF_PARTIAL_BIT) : 0x7fffffff; }
+    if ((uses & 1) && ++i0 < L.n0) raw0 = L.entry(0, i0);
+    if ((uses & 2) && ++i1 < L.n1) raw1 = L.entry(1, i1);
     return true;
   }
 };
@@ -300,21 +304,19 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       for (int u = 0; has_cur; ++u) {
         const bool has_nxt = mg.next(L, nxt_tile, nxt_uses);
         const int vs = u % C::NV, ksn = (u + 1) % C::NK;
-        bool v_ready = false, k_ready = false;
+        // the TMA barriers first: their data has normally landed long ago, and checking them here
+        // keeps them out of the gap between a stream's P arriving and its MMAs being issued
+        mbar_wait(bar(C::B_VF + vs), (u / C::NV) & 1, wc);
+        if (has_nxt) mbar_wait(bar(C::B_KF + ksn), ((u + 1) / C::NK) & 1, wc);
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
           if (cur_uses & (1 << j)) {
             mbar_wait(bar(C::B_PF + j), pv_cnt[j] & 1, wc);
-            if (!v_ready) { mbar_wait(bar(C::B_VF + vs), (u / C::NV) & 1, wc); v_ready = true; }
             tc_fence_after();
             issue_pv(j, vs, pv_cnt[j] == 0);
             ++pv_cnt[j];
           }
-          if (has_nxt && (nxt_uses & (1 << j))) {
-            if (!k_ready) { mbar_wait(bar(C::B_KF + ksn), ((u + 1) / C::NK) & 1, wc); k_ready = true; }
-            tc_fence_after();
-            issue_s(j, ksn);
-          }
+          if (has_nxt && (nxt_uses & (1 << j))) issue_s(j, ksn);
         }
         tc_commit(bar(C::B_VE + vs));
         if (has_nxt) tc_commit(bar(C::B_KE + ksn));

@@ -29,6 +29,10 @@ from paper_2505_21036_b200 import synth  # noqa: E402
 METRIC = "dense_equiv_tflops_sparse_attn"
 UNIT = "TFLOP/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one rf_attn_kernel launch, from single-pass ncu captures
+# (profiles/rf_attn_kernel_hunyuan720p_dram_bytes.md); None where no capture exists.
+ATTN_DRAM_BYTES = {"hunyuan720p": 4.21e9, "sweep_33x3600": 4.21e9, "sweep_16x2040": 0.733e9}
+
 
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -271,7 +275,7 @@ def run_cuda(args, wl):
                        "L_text": wl.L_text, "N": wl.N, "block": 128, "temporal_permute": 1,
                        "frame_window": wl.frame_window, "spatial_window": wl.spatial_window,
                        "textural_stride": wl.textural_stride, "sample_stride": wl.sample_stride,
-                       "l2": "inputs (2.2 GB of Q/K/V) exceed L2", "parallelism": f"replicas x{world}"},
+                       "l2": f"inputs ({3 * wl.B * wl.H * wl.N * wl.D * 2 / 1e9:.2f} GB of Q/K/V) exceed the 126 MB L2; no flush", "parallelism": f"replicas x{world}"},
             "clocks": clocks,
             "e2e": {"value": dist_util.replica_throughput(dflops, e2e_ms, world) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": o.numel() * 2},
@@ -288,7 +292,9 @@ def run_cuda(args, wl):
             "dense_equiv_tflops_attn_call": dflops / (sparse_ms * 1e-3) / 1e12,
             "dense_baseline_tflops": (dflops / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
             "roofline": {"kernel": "rf_attn_kernel", "bound": "tensor", "achieved": achieved, "peak": pk["bf16_sustained"],
-                         "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"], "traffic": None,
+                         "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"], "traffic": ATTN_DRAM_BYTES.get(wl.name),
+                         "traffic_unit": "bytes per launch (ncu, dram read + write)",
+                         "algorithmic_bytes_per_launch": 4 * wl.B * wl.H * wl.N * wl.D * 2,
                          "peak_kind": f"bf16 sustained, of {pk['source']}", "frac_of_burst": achieved / pk["bf16_burst"],
                          "algorithmic_flops_per_launch": tile_flops},
         }
@@ -308,7 +314,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="hunyuan720p", choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--ref-rows", type=int, default=512, help="query rows per oracle sample")
+    ap.add_argument("--ref-rows", type=int, default=4096, help="query rows per oracle sample (about 10-20 s of CPU work)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
     ap.add_argument("--no-dense", dest="dense", action="store_false", help="skip the dense-baseline timing")
     args = ap.parse_args()

@@ -1,242 +1,309 @@
 // ARM: Adaptive Recognition Module (Sec. 3.3, Eq. 6, Algorithm 1).
 //
-// For a sample I of video tokens (the first frame, or every omega-th token) each CTA takes 128
-// sampled query rows and streams all sampled keys through shared memory in blocks of 64 (cp.async,
-// double-buffered): scores on the tensor cores (mma.sync m16n8k16 bf16, fp32 accumulate), online
-// softmax in fp32 with warp shuffles for the row maximum, and next to the total mass the masked
-// masses: the part of the row kept by the Temporal, the Spatial and (when recalls are wanted) the
-// Textural mask restricted to I.  A key block that lies wholly inside or outside a mask's band for
-// all 16 rows of a warp is settled per block (frames grow monotonically with the sample index, and
-// on the first-frame sample so do positions); only blocks a band edge crosses test per element.
-// The n x n score matrix is never written.  Per-row recalls go to scratch; a second kernel
-// averages them in a fixed order (deterministic) and takes Algorithm 1's decision.
-#include "rf_common.cuh"
+// The sampled score matrix S' = Q' K'^T / sqrt(d) is a dense contraction, so it runs on tcgen05 like the
+// attention kernel, minus everything that concerns V: one CTA takes two 128-row tiles of sampled queries
+// ("streams") of one head and walks all 128-key tiles of the sample.  Sampled rows are fetched straight
+// from Q and K by TMA through tensor maps whose row stride is omega tokens (no gather pass).  Warp roles:
+//   warps 0-3 / 4-7  softmax statistics of stream 0 / 1 (one thread per sampled query row)
+//   warp 8           TMA producer: both Q tiles once, then K tiles into a shared-memory ring
+//   warp 9           MMA issuer; each stream's S accumulator is double-buffered in TMEM (4 x 128 columns),
+//                    so the next tile's scores are computed while the current ones are being reduced
+// Per tile a softmax thread reads its row of S (tcgen05.ld), hands the buffer back, and updates an
+// online softmax (running maximum, total mass) plus the masked masses Algorithm 1 needs: the share of
+// the row kept by the sampled Temporal / Spatial (/ Textural, when recalls are requested) mask.
+// On the first-frame sample positions equal sample indices, and on the stride sample frames grow
+// with the sample index, so a row's kept keys form one index interval: tiles wholly inside or outside
+// it for all 32 rows of a warp cost nothing extra, tiles an edge crosses use a 128-bit keep word per
+// row.  Only the Temporal mask on the stride sample (RF_SAMPLE_GLOBAL) and the Textural diagnostic
+// need per-key attributes, computed cooperatively per tile.
+// Per-row recalls go to scratch; a second kernel averages them in a fixed order (deterministic) and
+// takes Algorithm 1's decision.  The n x n score matrix is never written.
+#include "rf_sm100.cuh"
 
 namespace {
 
-constexpr int ARM_ROWS = 128;  // query rows per CTA (16 per warp)
-constexpr int ARM_KEYS = 64;   // keys per shared-memory block
-constexpr int ARM_THREADS = 256;
+using namespace sm100;
 
-// Which masked masses a launch accumulates.
-constexpr int ARM_LOCAL_T = 0;    // first-frame sample: Temporal only (positions = sample index)
-constexpr int ARM_GLOBAL_S = 1;   // stride sample: Spatial
-constexpr int ARM_GLOBAL_ST = 2;  // stride sample: Spatial and Temporal
+constexpr int ARM_TILE = 128;
+constexpr int ARM_THREADS = 384;           // softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
+constexpr int ARM_TMA_WARP = 8, ARM_MMA_WARP = 9;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+struct ArmMaps { CUtensorMap q[2], k[2]; };   // per sample: 0 = stride sample, 1 = first-frame sample
 
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
+struct ArmSample {
+  int n;          // sampled tokens
+  int stride;     // token index of sample m is m * stride
+  int pairs;      // CTAs per head: ceil(ceil(n/128) / 2)
+  int want_t;     // accumulate the Temporal mass on this sample
+  int want_s;     // accumulate the Spatial mass on this sample
+  float* out;     // [B*H][3][n_pad]
+};
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// 16-byte asynchronous copy; zero-fills when !valid (src must still be a readable address).
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-  const int sz = valid ? 16 : 0;
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+template <int D>
+struct ArmCfg {
+  static constexpr int KB = (D + 63) / 64;
+  static constexpr int COL1 = D - 64;
+  static constexpr uint32_t BLK = 128 * 128;
+  static constexpr uint32_t TILE = KB * BLK;
+  static constexpr int NK = D == 64 ? 6 : 4;
+  static constexpr uint32_t Q = 0;
+  static constexpr uint32_t K0 = Q + 2 * TILE;
+  static constexpr uint32_t BAR = K0 + NK * TILE;
+  static constexpr int B_Q = 0, B_KF = 1, B_KE = B_KF + NK, B_SF = B_KE + NK, B_SE = B_SF + 4, B_COUNT = B_SE + 4;
+  static constexpr uint32_t MISC = BAR + 8 * ((B_COUNT + 7) / 8 * 8);
+  static constexpr uint32_t ATTR = MISC + 64;                    // int [8 warps][2][128]: key position / checkerboard flag
+  static constexpr uint32_t TOTAL = ATTR + 8 * 2 * 128 * 4;
+  static constexpr uint32_t ALLOC = TOTAL + 1024;
+  static_assert(ALLOC <= 227 * 1024, "exceeds the shared memory a CTA can opt in to");
+  static __host__ __device__ constexpr uint32_t koff(int ks) {
+    return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks * 16 - COL1) * 2u;
+  }
+};
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-
-struct KeyAttr { int f, p, c; };  // frame, in-frame position, 1 if in the checkerboard set C
-
-__device__ __forceinline__ KeyAttr token_attr(const RfGeom& g, int tok) {
-  KeyAttr a;
-  a.f = tok / g.S;
-  a.p = tok - a.f * g.S;
-  const int y = a.p / g.Wf, x = a.p - y * g.Wf;
-  a.c = (y % g.tau) == (x % g.tau);
-  return a;
+__device__ __forceinline__ uint32_t bits_below(int n) { return n >= 32 ? 0xffffffffu : ((1u << n) - 1u); }
+// Bits of the tile starting at key u0 that fall in the key interval [a, b).
+__device__ __forceinline__ void interval_bits(uint32_t (&w)[4], int u0, int a, int b) {
+  a = max(a - u0, 0);
+  b = min(b - u0, ARM_TILE);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int lo = min(max(a - 32 * k, 0), 32), hi = min(max(b - 32 * k, 0), 32);
+    w[k] = hi > lo ? (bits_below(hi) & ~bits_below(lo)) : 0u;
+  }
 }
 
-// 0: no pair of (rows, cols) within w, 2: every pair within w, 1: mixed.  Closed integer ranges.
-__device__ __forceinline__ int band_class(int ra, int rb, int ca, int cb, int w) {
-  const int dmin = max(max(ca - rb, ra - cb), 0), dmax = max(rb - ca, cb - ra);
-  return dmax <= w ? 2 : (dmin > w ? 0 : 1);
-}
+template <int D, bool TEX>
+__global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_constant__ ArmMaps maps, const RfGeom g,
+                                                                const ArmSample sm0, const ArmSample sm1, int n_pad,
+                                                                float scale_log2, int32_t* dev_status) {
+  using C = ArmCfg<D>;
+  constexpr uint32_t IDESC_S = idesc_bf16(128, 128, 0);
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  auto bar = [&](int slot) -> uint32_t { return base + C::BAR + 8u * slot; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + C::MISC);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::MISC + 8);
 
-// grid = (ceil(n/128), B*H).  stride: token index of sample m is m*stride.
-// row_out: [B*H][3][n_pad] per-row recalls (temporal, spatial, textural) of this sample; only the
-// masses this launch accumulates are written.
-template <int D, int MODE, bool TEX>
-__global__ void __launch_bounds__(ARM_THREADS) rf_arm_rows_kernel(RfGeom g, int n, int stride, int n_pad,
-                                                                   const __nv_bfloat16* __restrict__ q,
-                                                                   const __nv_bfloat16* __restrict__ k,
-                                                                   float scale_log2, float* __restrict__ row_out) {
-  constexpr int LD = D + 8;  // padded row, keeps ldmatrix conflict-free
-  constexpr int VEC = D / 8;
-  constexpr bool WANT_T = MODE != ARM_GLOBAL_S, WANT_S = MODE != ARM_LOCAL_T;
-  constexpr bool T_BAND = MODE == ARM_LOCAL_T;  // Temporal mask is a band in sample-index space
-  // the Q tile first; once its fragments are in registers the same memory holds two key blocks
-  __shared__ __align__(16) __nv_bfloat16 buf[ARM_ROWS * LD];
-  __shared__ int kf[2][ARM_KEYS], kp[2][ARM_KEYS], kc[2][ARM_KEYS];
-
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = blockIdx.y;
-  const int row0 = blockIdx.x * ARM_ROWS;
-  const size_t head = (size_t)bh * g.N * D;
+  // blockIdx.x enumerates the CTAs of the stride sample first, then those of the first-frame sample
+  const bool second = (int)blockIdx.x >= sm0.pairs;
+  const ArmSample& sm = second ? sm1 : sm0;
+  const int which = second ? 1 : 0;
+  const int pair = second ? blockIdx.x - sm0.pairs : blockIdx.x;
+  const int n = sm.n, stride = sm.stride;
+  const int nt = rf_cdiv(n, ARM_TILE);
+  const int qt0 = 2 * pair;
+  const bool stream1 = qt0 + 1 < nt;
+  const CUtensorMap* map_q = &maps.q[which];
+  const CUtensorMap* map_k = &maps.k[which];
+  const bool t_band = sm.want_t && stride == 1;       // positions = sample indices: the Temporal mask is one interval
+  const bool t_generic = sm.want_t && stride != 1;    // needs per-key positions
 
-  for (int i = tid; i < ARM_ROWS * VEC; i += ARM_THREADS) {
-    const int r = i / VEC, c = i % VEC;
-    const int m = min(row0 + r, n - 1);
-    cp_async16(smem_u32(&buf[r * LD + c * 8]), q + head + (size_t)m * stride * D + c * 8, true);
+  if (tid == 0) {
+    mbar_init(bar(C::B_Q), 1);
+    for (int s = 0; s < C::NK; ++s) { mbar_init(bar(C::B_KF + s), 1); mbar_init(bar(C::B_KE + s), 1); }
+    for (int s = 0; s < 4; ++s) { mbar_init(bar(C::B_SF + s), 1); mbar_init(bar(C::B_SE + s), 4); }
+    *abort_flag = 0;
+    mbar_init_fence();
   }
-  cp_async_commit();
-  cp_async_wait<0>();
+  if (warp == ARM_TMA_WARP) {
+    if (lane == 0) { prefetch_tmap(map_q); prefetch_tmap(map_k); }
+    __syncwarp();
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  }
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const WaitCtx wc{abort_flag, dev_status};
 
-  uint32_t qa[D / 16][4];
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    if (warp == ARM_TMA_WARP) {
+      if (lane == 0) {
+        mbar_expect_tx(bar(C::B_Q), 2 * C::TILE);
 #pragma unroll
-  for (int ks = 0; ks < D / 16; ++ks) {
-    const uint32_t addr = smem_u32(&buf[(warp * 16 + (lane & 15)) * LD + ks * 16 + (lane >> 4) * 8]);
-    ldmatrix_x4(addr, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
-  }
-  __syncthreads();  // every warp has its fragments: the buffer may be overwritten with keys
-
-  auto load_keys = [&](int blk) {
-    const int k0 = blk * ARM_KEYS, b = blk & 1;
-    for (int i = tid; i < ARM_KEYS * VEC; i += ARM_THREADS) {
-      const int r = i / VEC, c = i % VEC;
-      const int m = k0 + r;
-      cp_async16(smem_u32(&buf[(b * ARM_KEYS + r) * LD + c * 8]), k + head + (size_t)min(m, n - 1) * stride * D + c * 8, m < n);
-    }
-    if (tid < ARM_KEYS) {
-      const KeyAttr a = token_attr(g, min(k0 + tid, n - 1) * stride);
-      kf[b][tid] = a.f; kp[b][tid] = a.p; kc[b][tid] = a.c;
-    }
-    cp_async_commit();
-  };
-
-  // the two rows this thread sees: warp*16 + lane/4 and +8
-  int rf[2], rp[2];
+        for (int j = 0; j < 2; ++j)
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const KeyAttr a = token_attr(g, min(row0 + warp * 16 + (lane >> 2) + h * 8, n - 1) * stride);
-    rf[h] = a.f;
-    rp[h] = a.p;
-  }
-  // row range of this warp, for the per-block band classification
-  const int wra = min(row0 + warp * 16, n - 1), wrb = min(row0 + warp * 16 + 15, n - 1);
-  const int wfa = (wra * stride) / g.S, wfb = (wrb * stride) / g.S;
-
-  float mx[2] = {-INFINITY, -INFINITY};
-  float l_all[2] = {0.f, 0.f}, l_t[2] = {0.f, 0.f}, l_s[2] = {0.f, 0.f}, l_c[2] = {0.f, 0.f};
-
-  const int nblk = rf_cdiv(n, ARM_KEYS);
-  load_keys(0);
-  for (int blk = 0; blk < nblk; ++blk) {
-    const int k0 = blk * ARM_KEYS, b = blk & 1;
-    if (blk + 1 < nblk) {
-      load_keys(blk + 1);
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
-    __syncthreads();
-    const __nv_bfloat16* Ks = buf + b * ARM_KEYS * LD;
-
-    float acc[ARM_KEYS / 8][4];
+          for (int kb = 0; kb < C::KB; ++kb)
+            tma_load_3d(base + C::Q + j * C::TILE + kb * C::BLK, map_q, kb * C::COL1, (qt0 + j) * ARM_TILE, bh, bar(C::B_Q));
+        for (int u = 0; u < nt; ++u) {
+          const int ks = u % C::NK;
+          if (u >= C::NK) mbar_wait(bar(C::B_KE + ks), ((u / C::NK) - 1) & 1, wc);
+          mbar_expect_tx(bar(C::B_KF + ks), C::TILE);
 #pragma unroll
-    for (int nt = 0; nt < ARM_KEYS / 8; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+          for (int kb = 0; kb < C::KB; ++kb)
+            tma_load_3d(base + C::K0 + ks * C::TILE + kb * C::BLK, map_k, kb * C::COL1, u * ARM_TILE, bh, bar(C::B_KF + ks));
+        }
+      }
+    } else if (warp == ARM_MMA_WARP) {
+      if (lane == 0) {
+        constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+        auto desc = [](uint32_t lo) -> uint64_t { return ((uint64_t)DESC_HI << 32) | lo; };
+        const uint32_t q_lo = ((base + C::Q) >> 4) | (1u << 16), k_lo = ((base + C::K0) >> 4) | (1u << 16);
+        mbar_wait(bar(C::B_Q), 0, wc);
+        for (int u = 0; u < nt; ++u) {
+          const int ks = u % C::NK, b = u & 1;
+          mbar_wait(bar(C::B_KF + ks), (u / C::NK) & 1, wc);
 #pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
+          for (int j = 0; j < 2; ++j) {
+            if (j == 1 && !stream1) continue;
+            if (u >= 2) mbar_wait(bar(C::B_SE + j * 2 + b), ((u >> 1) - 1) & 1, wc);
+            tc_fence_after();
+            const uint32_t a0 = q_lo + j * (C::TILE >> 4), b0 = k_lo + ks * (C::TILE >> 4);
 #pragma unroll
-      for (int np = 0; np < ARM_KEYS / 16; ++np) {
-        const int mi = lane >> 3;
-        const uint32_t addr = smem_u32(&Ks[(np * 16 + (mi >> 1) * 8 + (lane & 7)) * LD + ks * 16 + (mi & 1) * 8]);
-        uint32_t b0, b1, b2, b3;
-        ldmatrix_x4(addr, b0, b1, b2, b3);
-        mma_bf16_16816(acc[np * 2], qa[ks], b0, b1);
-        mma_bf16_16816(acc[np * 2 + 1], qa[ks], b2, b3);
+            for (int k = 0; k < D / 16; ++k)
+              mma_ss(tmem_base + (j * 2 + b) * 128, desc(a0 + (C::koff(k) >> 4)), desc(b0 + (C::koff(k) >> 4)), IDESC_S, k > 0);
+            tc_commit(bar(C::B_SF + j * 2 + b));
+          }
+          tc_commit(bar(C::B_KE + ks));
+        }
       }
     }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    const int j = warp >> 2;
+    if (j == 0 || stream1) {
+      const int m = (qt0 + j) * ARM_TILE + (tid & 127);          // sampled row of this thread
+      const int mc = min(m, n - 1);
+      const int tok = mc * stride;
+      const int rf = tok / g.S, rp = tok - rf * g.S;
+      // kept key intervals of this row, in sample-index space
+      const int t_lo = rp - g.ws, t_hi = rp + g.ws + 1;                               // first-frame sample only
+      const int s_lo = rf_cdiv(max(rf - g.wf, 0) * g.S, stride);
+      const int s_hi = rf_cdiv((rf + g.wf + 1) * g.S, stride);                         // exclusive
+      const uint32_t t_s = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + j * 256;
+      int* attr_p = reinterpret_cast<int*>(base_ptr + C::ATTR) + warp * 256;           // per-warp tables
+      int* attr_c = attr_p + 128;
+      float mx = -INFINITY, l_all = 0.f, l_t = 0.f, l_s = 0.f, l_c = 0.f;
 
-    // key slots past the sample (last block only) carry -inf
-    if (k0 + ARM_KEYS > n) {
-#pragma unroll
-      for (int nt = 0; nt < ARM_KEYS / 8; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if (k0 + nt * 8 + (lane & 3) * 2 + (e & 1) >= n) acc[nt][e] = -INFINITY;
-    }
-    float bm[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int nt = 0; nt < ARM_KEYS / 8; ++nt) {
-      bm[0] = fmaxf(bm[0], fmaxf(acc[nt][0], acc[nt][1]));
-      bm[1] = fmaxf(bm[1], fmaxf(acc[nt][2], acc[nt][3]));
-    }
-    float neg_m[2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      bm[h] = fmaxf(bm[h], __shfl_xor_sync(0xffffffffu, bm[h], 1));
-      bm[h] = fmaxf(bm[h], __shfl_xor_sync(0xffffffffu, bm[h], 2));
-      const float m_new = fmaxf(mx[h], bm[h] * scale_log2);   // finite: every block holds >= 1 real key
-      const float corr = ex2f(mx[h] - m_new);                  // 0 on the first block
-      l_all[h] *= corr; l_t[h] *= corr; l_s[h] *= corr; l_c[h] *= corr;
-      mx[h] = m_new;
-      neg_m[h] = -m_new;
-    }
+      for (int u = 0; u < nt; ++u) {
+        const int b = u & 1, u0 = u * ARM_TILE;
+        mbar_wait(bar(C::B_SF + j * 2 + b), (u >> 1) & 1, wc);
+        tc_fence_after();
+        uint32_t s[128];
+        {
+          uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+          uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+          uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+          uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+          tmem_ld32(t_s + b * 128, s0);
+          tmem_ld32(t_s + b * 128 + 32, s1);
+          tmem_ld32(t_s + b * 128 + 64, s2);
+          tmem_ld32(t_s + b * 128 + 96, s3);
+          tc_wait_ld();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C::B_SE + j * 2 + b));   // the buffer may be refilled
 
-    // band classes of this block for the warp's 16 rows (warp-uniform)
-    const int ca = k0, cb = min(k0 + ARM_KEYS - 1, n - 1);
-    const int t_cls = !WANT_T ? 0 : (T_BAND ? band_class(wra, wrb, ca, cb, g.ws) : 1);
-    const int s_cls = !WANT_S ? 0 : band_class(wfa, wfb, (ca * stride) / g.S, (cb * stride) / g.S, g.wf);
+        if (u0 + ARM_TILE > n) {                                 // keys past the sample
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (u0 + c >= n) s[c] = 0xff800000u;
+        }
+        float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 128; c += 4) {
+          m0 = fmaxf(m0, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
+          m1 = fmaxf(m1, fmaxf(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])));
+        }
+        const float m_new = fmaxf(mx, fmaxf(m0, m1) * scale_log2);   // finite: every tile holds a real key
+        const float corr = ex2f(mx - m_new);
+        l_all *= corr; l_t *= corr; l_s *= corr; l_c *= corr;
+        mx = m_new;
 
-    float bs[2] = {0.f, 0.f}, bt[2] = {0.f, 0.f}, bsp[2] = {0.f, 0.f}, bc[2] = {0.f, 0.f};
+        // where does this tile lie relative to the row's kept intervals?  0 outside, 2 inside, 1 crossing
+        const int u1 = min(u0 + ARM_TILE, n);
+        int t_cls = 0, s_cls = 0;
+        if (t_band) {
+          const bool in = t_lo <= u0 && u1 <= t_hi, out = u1 <= t_lo || t_hi <= u0;
+          t_cls = __all_sync(0xffffffffu, in) ? 2 : (__all_sync(0xffffffffu, out) ? 0 : 1);
+        } else if (t_generic) {
+          t_cls = 1;
+        }
+        if (sm.want_s) {
+          const bool in = s_lo <= u0 && u1 <= s_hi, out = u1 <= s_lo || s_hi <= u0;
+          s_cls = __all_sync(0xffffffffu, in) ? 2 : (__all_sync(0xffffffffu, out) ? 0 : 1);
+        }
+        const float2 sc2 = make_float2(scale_log2, scale_log2), mneg = make_float2(-m_new, -m_new);
+        if (!TEX && t_cls != 1 && s_cls != 1) {
+          float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int nt = 0; nt < ARM_KEYS / 8; ++nt) {
+          for (int c = 0; c < 128; c += 4) {
+            float2 e0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, mneg);
+            float2 e1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, mneg);
+            e0.x = ex2f(e0.x); e0.y = ex2f(e0.y);
+            e1.x = ex2f(e1.x); e1.y = ex2f(e1.y);
+            la = __fadd2_rn(la, e0);
+            lb = __fadd2_rn(lb, e1);
+          }
+          const float bs = (la.x + la.y) + (lb.x + lb.y);
+          l_all += bs;
+          if (t_cls == 2) l_t += bs;
+          if (s_cls == 2) l_s += bs;
+        } else {
+          // keep words per mask for this row and tile
+          uint32_t wt[4] = {0, 0, 0, 0}, ws[4] = {0, 0, 0, 0}, wx[4] = {0, 0, 0, 0};
+          if (t_band) interval_bits(wt, u0, t_lo, t_hi);
+          if (sm.want_s) interval_bits(ws, u0, s_lo, s_hi);
+          if (TEX || t_generic) {
+            // per-key attributes of the tile, four keys per lane, into this warp's table
+            __syncwarp();
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int h = e >> 1;
-        const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
-        const float p = ex2f(fmaf(acc[nt][e], scale_log2, neg_m[h]));
-        bs[h] += p;
-        if (WANT_T && t_cls == 1) { if (abs(kp[b][col] - rp[h]) <= g.ws) bt[h] += p; }
-        if (WANT_S && s_cls == 1) { if (abs(kf[b][col] - rf[h]) <= g.wf) bsp[h] += p; }
-        if (TEX) { if (kc[b][col]) bc[h] += p; }
+            for (int i = 0; i < 4; ++i) {
+              const int c = lane * 4 + i;
+              const int ktok = min(u0 + c, n - 1) * stride;
+              const int kp = ktok % g.S;
+              const int y = kp / g.Wf, x = kp - y * g.Wf;
+              attr_p[c] = kp;
+              attr_c[c] = (y % g.tau) == (x % g.tau);
+            }
+            __syncwarp();
+#pragma unroll 4
+            for (int c = 0; c < 128; ++c) {
+              if (t_generic) { const int dp = attr_p[c] - rp; if ((dp < 0 ? -dp : dp) <= g.ws) wt[c >> 5] |= 1u << (c & 31); }
+              if (TEX && attr_c[c]) wx[c >> 5] |= 1u << (c & 31);
+            }
+          }
+          float bs = 0.f, bt = 0.f, bsp = 0.f, bx = 0.f;
+#pragma unroll
+          for (int c = 0; c < 128; ++c) {
+            const float p = ex2f(fmaf(__uint_as_float(s[c]), scale_log2, -m_new));
+            bs += p;
+            if ((wt[c >> 5] >> (c & 31)) & 1u) bt += p;
+            if ((ws[c >> 5] >> (c & 31)) & 1u) bsp += p;
+            if (TEX) { if ((wx[c >> 5] >> (c & 31)) & 1u) bx += p; }
+          }
+          l_all += bs;
+          l_t += bt;
+          l_s += bsp;
+          l_c += bx;
+        }
+      }
+      if (m < n) {
+        float* out = sm.out + (size_t)bh * 3 * n_pad;
+        const float inv = 1.f / l_all;
+        if (sm.want_t) out[m] = l_t * inv;
+        if (sm.want_s) out[n_pad + m] = l_s * inv;
+        if (TEX) out[2 * n_pad + m] = l_c * inv;
       }
     }
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      l_all[h] += bs[h];
-      if (WANT_T) l_t[h] += t_cls == 2 ? bs[h] : bt[h];
-      if (WANT_S) l_s[h] += s_cls == 2 ? bs[h] : bsp[h];
-      if (TEX) l_c[h] += bc[h];
-    }
-    __syncthreads();  // block consumed: its buffer is the target of the next prefetch
   }
 
-  // quad reduction of the partial masses, then one lane per row writes its recalls
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-#pragma unroll
-    for (int o = 1; o <= 2; o <<= 1) {
-      l_all[h] += __shfl_xor_sync(0xffffffffu, l_all[h], o);
-      l_t[h] += __shfl_xor_sync(0xffffffffu, l_t[h], o);
-      l_s[h] += __shfl_xor_sync(0xffffffffu, l_s[h], o);
-      l_c[h] += __shfl_xor_sync(0xffffffffu, l_c[h], o);
-    }
-    const int m = row0 + warp * 16 + (lane >> 2) + h * 8;
-    if ((lane & 3) == 0 && m < n) {
-      float* out = row_out + (size_t)bh * 3 * n_pad;
-      const float inv = 1.f / l_all[h];
-      if (WANT_T) out[m] = l_t[h] * inv;
-      if (WANT_S) out[n_pad + m] = l_s[h] * inv;
-      if (TEX) out[2 * n_pad + m] = l_c[h] * inv;
-    }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == ARM_TMA_WARP) {
+    if (*abort_flag) __nanosleep(20000);
+    __syncwarp();
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -272,32 +339,30 @@ __global__ void __launch_bounds__(256) rf_arm_decide_kernel(int n_loc, int n_glb
   }
 }
 
-template <int D, int MODE, bool TEX>
-cudaError_t launch_rows(const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q, const __nv_bfloat16* k,
-                        float* out, cudaStream_t st) {
-  dim3 grid(rf_cdiv(n, ARM_ROWS), g.B * g.H);
+template <int D, bool TEX>
+cudaError_t launch_arm_t(const ArmMaps& maps, const RfGeom& g, const ArmSample& s0, const ArmSample& s1, int n_pad,
+                         int32_t* dev_status, cudaStream_t st) {
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    e = cudaFuncSetAttribute(rf_arm_kernel<D, TEX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ArmCfg<D>::ALLOC);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  dim3 grid(s0.pairs + s1.pairs, g.B * g.H);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
-  rf_arm_rows_kernel<D, MODE, TEX><<<grid, ARM_THREADS, 0, st>>>(g, n, stride, n_pad, q, k, scale_log2, out);
+  rf_arm_kernel<D, TEX><<<grid, ARM_THREADS, ArmCfg<D>::ALLOC, st>>>(maps, g, s0, s1, n_pad, scale_log2, dev_status);
   return cudaGetLastError();
 }
 
-template <int D>
-cudaError_t launch_rows_m(int mode, bool tex, const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q,
-                          const __nv_bfloat16* k, float* out, cudaStream_t st) {
-  if (mode == ARM_LOCAL_T) return launch_rows<D, ARM_LOCAL_T, false>(g, n, stride, n_pad, q, k, out, st);
-  if (mode == ARM_GLOBAL_S)
-    return tex ? launch_rows<D, ARM_GLOBAL_S, true>(g, n, stride, n_pad, q, k, out, st)
-               : launch_rows<D, ARM_GLOBAL_S, false>(g, n, stride, n_pad, q, k, out, st);
-  return tex ? launch_rows<D, ARM_GLOBAL_ST, true>(g, n, stride, n_pad, q, k, out, st)
-             : launch_rows<D, ARM_GLOBAL_ST, false>(g, n, stride, n_pad, q, k, out, st);
-}
-
-cudaError_t launch_rows_d(int mode, bool tex, const RfGeom& g, int n, int stride, int n_pad, const __nv_bfloat16* q,
-                          const __nv_bfloat16* k, float* out, cudaStream_t st) {
+cudaError_t launch_arm_d(bool tex, const ArmMaps& maps, const RfGeom& g, const ArmSample& s0, const ArmSample& s1,
+                         int n_pad, cudaStream_t st) {
   switch (g.D) {
-    case 64: return launch_rows_m<64>(mode, tex, g, n, stride, n_pad, q, k, out, st);
-    case 96: return launch_rows_m<96>(mode, tex, g, n, stride, n_pad, q, k, out, st);
-    case 128: return launch_rows_m<128>(mode, tex, g, n, stride, n_pad, q, k, out, st);
+    case 64: return tex ? launch_arm_t<64, true>(maps, g, s0, s1, n_pad, nullptr, st) : launch_arm_t<64, false>(maps, g, s0, s1, n_pad, nullptr, st);
+    case 96: return tex ? launch_arm_t<96, true>(maps, g, s0, s1, n_pad, nullptr, st) : launch_arm_t<96, false>(maps, g, s0, s1, n_pad, nullptr, st);
+    case 128: return tex ? launch_arm_t<128, true>(maps, g, s0, s1, n_pad, nullptr, st) : launch_arm_t<128, false>(maps, g, s0, s1, n_pad, nullptr, st);
   }
   return cudaErrorInvalidValue;
 }
@@ -321,14 +386,23 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
   float* rows_loc = row_scratch + (size_t)g.B * g.H * 3 * n_pad;
   const bool alg1 = sample_mode == RF_SAMPLE_ALG1;
   const bool tex = recall != nullptr;   // the Textural recall is a diagnostic: Algorithm 1 does not use it
-  cudaError_t e = launch_rows_d(alg1 ? ARM_GLOBAL_S : ARM_GLOBAL_ST, tex, g, n_glb, omega, n_pad, q, k, rows_glb, st);
+  const int heads = g.B * g.H;
+  const size_t row_bytes = (size_t)g.D * 2, head_bytes = (size_t)g.N * g.D * 2;
+  ArmMaps maps;
+  bool ok = rf_encode_rows_map(&maps.q[0], q, g.D, n_glb, row_bytes * omega, head_bytes, heads) &&
+            rf_encode_rows_map(&maps.k[0], k, g.D, n_glb, row_bytes * omega, head_bytes, heads) &&
+            rf_encode_rows_map(&maps.q[1], q, g.D, n_loc, row_bytes, head_bytes, heads) &&
+            rf_encode_rows_map(&maps.k[1], k, g.D, n_loc, row_bytes, head_bytes, heads);
+  if (!ok) return cudaErrorUnknown;
+  ArmSample s0, s1;
+  s0.n = n_glb; s0.stride = omega; s0.pairs = rf_cdiv(rf_cdiv(n_glb, ARM_TILE), 2);
+  s0.want_t = alg1 ? 0 : 1; s0.want_s = 1; s0.out = rows_glb;
+  s1.n = n_loc; s1.stride = 1; s1.pairs = alg1 ? rf_cdiv(rf_cdiv(n_loc, ARM_TILE), 2) : 0;
+  s1.want_t = 1; s1.want_s = 0; s1.out = rows_loc;
+  cudaError_t e = launch_arm_d(tex, maps, g, s0, s1, n_pad, st);
   if (e != cudaSuccess) return e;
-  if (alg1) {
-    e = launch_rows_d(ARM_LOCAL_T, false, g, n_loc, 1, n_pad, q, k, rows_loc, st);
-    if (e != cudaSuccess) return e;
-  }
-  rf_arm_decide_kernel<<<g.B * g.H, 256, 0, st>>>(n_loc, n_glb, n_pad, sample_mode, alpha, rows_loc, rows_glb,
-                                                  head_class, recall);
+  rf_arm_decide_kernel<<<heads, 256, 0, st>>>(n_loc, n_glb, n_pad, sample_mode, alpha, rows_loc, rows_glb, head_class,
+                                              recall);
   return cudaGetLastError();
 }
 

@@ -44,6 +44,10 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
                           const __nv_bfloat16* k, int32_t* head_class, float* recall, float* row_scratch,
                           cudaStream_t st);
 size_t rf_arm_scratch_floats(const RfGeom& g, int omega);
+// Tensor map over bf16 rows: [heads][rows][D] with the given row and head strides in bytes (multiples of 16),
+// box = 64 columns x 128 rows, 128-byte swizzle, zero fill past `rows`.
+bool rf_encode_rows_map(CUtensorMap* m, const void* ptr, int D, int rows, size_t row_stride_bytes,
+                        size_t head_stride_bytes, int heads);
 // Validates shape and parameters as the entry points do and fills the kernel-side geometry.
 rf_status rf_checked_geom(const rf_shape* shape, const rf_params* params, RfGeom* out);
 

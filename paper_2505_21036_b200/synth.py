@@ -92,6 +92,11 @@ WORKLOADS: Dict[str, Workload] = {
     "cogvideox": _wl("cogvideox", 2, 1, 48, 64, 13, 30, 45, 226, mode=0, omega=15, amp=0.5),
     # same shape, planted amplitude strong enough that all three branches fire
     "cogvideox_cal": _wl("cogvideox_cal", 2, 1, 48, 64, 13, 30, 45, 226, mode=0, omega=15, amp=2.0),
+    # parameter-sensitivity settings on the CogVideoX-shaped layer: bandwidth 0.18 / 0.13, stride 3 / 4
+    "cogvideox_2p5x": _wl("cogvideox_2p5x", 2, 1, 48, 64, 13, 30, 45, 226, wf=int(0.18 * 13), ws=int(0.18 * 1350), tau=3,
+                          mode=0, omega=15, amp=2.0),
+    "cogvideox_3p0x": _wl("cogvideox_3p0x", 2, 1, 48, 64, 13, 30, 45, 226, wf=int(0.13 * 13), ws=int(0.13 * 1350), tau=4,
+                          mode=0, omega=15, amp=2.0),
     # OpenSoraPlan-1.2-shaped layer; 1 % of tokens sampled at equal intervals
     "opensoraplan": _wl("opensoraplan", 3, 1, 24, 96, 24, 45, 80, 300, mode=1, omega=100, amp=1.5),
     # HunyuanVideo-720p-shaped layer

@@ -143,3 +143,24 @@ def test_pattern_mix_sweep(name):
             check_lists(run, classes, sample_tiles(run.sched.nQ, k=3), heads=[0, 1, 2])
             O, lse = gpu_outputs(run)
             check_rows(run, O, lse, classes, rows, [0, H // 2 + 1, H - 1])
+
+
+@pytest.mark.parametrize("name", ["cogvideox_2p5x", "cogvideox_3p0x"])
+def test_sensitivity_settings(name):
+    """Bandwidth 0.18 / 0.13 with checkerboard stride 3 / 4 (the 2.5x and 3.0x settings): general tau, narrow
+    windows, forced even mix so that every pattern is exercised whatever ARM decides."""
+    wl = synth.WORKLOADS[name]
+    run = gu.Run(wl, qkv=inputs(name))
+    classes = [S_, T_, X_] * (wl.H // 3)
+    run.force_classes(classes)
+    run.build()
+    check_lists(run, classes, None, heads=[0, 1, 2])
+    O, lse = gpu_outputs(run)
+    check_rows(run, O, lse, classes, synth.sample_rows(wl, 256, seed=8), range(0, wl.H, 5))
+    # kept compute against the closed forms: band 1-(1-b)^2, checkerboard ~1/tau (video x video part)
+    g = gu.geom(wl)
+    cnt = run.sched.count.cpu().numpy()[0]
+    dens = cnt.sum(axis=1) / float(run.sched.nQ * run.sched.nKmax)
+    b = 0.18 if name.endswith("2p5x") else 0.13
+    assert abs(dens[2] - 1.0 / wl.textural_stride) < 0.03
+    assert dens[0] < 1 - (1 - b) ** 2 + 0.12 and dens[1] < 1 - (1 - b) ** 2 + 0.12

@@ -200,6 +200,53 @@ def arm_classify(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, pp: Patter
 
 
 # ----------------------------------------------------------------------------------------
+# RainFusion+ : per-head bandwidth (Sec. 4.3, "Qualitative Analysis and Integrability")
+# ----------------------------------------------------------------------------------------
+
+def windows_of(bandwidth: float, g: Geometry) -> Tuple[int, int]:
+    """(w_f, w_s) of a bandwidth b: floor(b*T) frames, floor(b*S) in-frame positions."""
+    return int(math.floor(bandwidth * g.T)), int(math.floor(bandwidth * g.S))
+
+
+def decide_plus(R_temporal: Sequence[float], R_spatial: Sequence[float], alpha: float) -> Tuple[int, int]:
+    """Recalls per candidate bandwidth (ascending).  The pattern is chosen as in Algorithm 1 (Temporal
+    first, then Spatial, else Textural), a pattern qualifying if ANY candidate reaches alpha; its
+    bandwidth is the smallest candidate that does.  Returns (class, candidate index or -1)."""
+    for cls, R in ((TEMPORAL, R_temporal), (SPATIAL, R_spatial)):
+        for i, r in enumerate(R):
+            if r >= alpha:
+                return cls, i
+    return TEXTURAL, -1
+
+
+def arm_head_plus(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, bandwidths: Sequence[float], tau: int,
+                  sample_mode: int, omega: int, alpha: float):
+    """ARM with dynamic bandwidth for one head: every candidate bandwidth's Temporal and Spatial recall on
+    the same approximate scores, then decide_plus.  Returns (class, index, window, R_t list, R_s list),
+    window = w_s of the chosen bandwidth for Temporal, w_f for Spatial, -1 for Textural."""
+    I_glb = global_sample(g, omega)
+    P_glb = approx_scores(q_bits, k_bits, I_glb)
+    if sample_mode == SAMPLE_ALG1:
+        I_t = local_sample(g)
+        P_t = approx_scores(q_bits, k_bits, I_t)
+    else:
+        I_t, P_t = I_glb, P_glb
+    R_t, R_s = [], []
+    for b in bandwidths:
+        wf, ws = windows_of(b, g)
+        pp = PatternParams(wf, ws, tau)
+        R_t.append(recall(P_t, keep_mask(TEMPORAL, I_t, I_t, g, pp)))
+        R_s.append(recall(P_glb, keep_mask(SPATIAL, I_glb, I_glb, g, pp)))
+    cls, idx = decide_plus(R_t, R_s, alpha)
+    window = -1
+    if cls == TEMPORAL:
+        window = windows_of(bandwidths[idx], g)[1]
+    elif cls == SPATIAL:
+        window = windows_of(bandwidths[idx], g)[0]
+    return cls, idx, window, R_t, R_s
+
+
+# ----------------------------------------------------------------------------------------
 # Head coordinate spaces, block masks and tile lists
 # ----------------------------------------------------------------------------------------
 

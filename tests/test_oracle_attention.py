@@ -221,3 +221,47 @@ def test_planted_heads_of_tiny_config_pick_their_patterns():
     a = orc.arm_head(q[0, 1, :64], k[0, 1, :64], g1, pp, orc.SAMPLE_ALG1, 1, 0.9)
     b = orc.arm_head(q[0, 1, :64], k[0, 1, :64], g1, pp, orc.SAMPLE_GLOBAL, 1, 0.9)
     assert a[1][0] == pytest.approx(b[1][0], abs=1e-14)
+
+
+# ---------------------------------------------------------------- RainFusion+ (dynamic bandwidth)
+
+@pytest.mark.parametrize("Rt,Rs,expect", [
+    ([0.5, 0.95, 0.99], [0.1, 0.2, 0.3], (TEMPORAL, 1)),      # smallest qualifying Temporal bandwidth
+    ([0.95, 0.96, 0.97], [0.99, 0.99, 0.99], (TEMPORAL, 0)),  # Temporal has priority even if Spatial is better
+    ([0.1, 0.2, 0.89], [0.2, 0.5, 0.9], (SPATIAL, 2)),        # >= alpha counts
+    ([0.1, 0.2, 0.3], [0.91, 0.95, 0.99], (SPATIAL, 0)),
+    ([0.1, 0.2, 0.3], [0.2, 0.5, 0.8999], (TEXTURAL, -1))])
+def test_dynamic_bandwidth_truth_table(Rt, Rs, expect):
+    assert orc.decide_plus(Rt, Rs, 0.9) == expect
+
+
+def test_windows_of_bandwidth():
+    g = Geometry(33, 45, 80, 256)
+    assert orc.windows_of(0.25, g) == (8, 900)
+    assert orc.windows_of(0.125, g) == (4, 450)
+    assert orc.windows_of(0.5, g) == (16, 1800)
+
+
+def test_dynamic_bandwidth_recalls_grow_with_the_window_and_match_the_fixed_bandwidth_path():
+    wl = synth.WORKLOADS["tiny"]
+    q, k, _ = synth.make_qkv(wl)
+    g = Geometry(wl.T, wl.frame_h, wl.frame_w, wl.L_text)
+    bws = [0.125, 0.25, 0.5]
+    for h in range(wl.H):
+        cls, idx, window, Rt, Rs = orc.arm_head_plus(q[0, h], k[0, h], g, bws, 2, orc.SAMPLE_ALG1, 4, 0.9)
+        assert all(a <= b + 1e-15 for a, b in zip(Rt, Rt[1:]))     # nested masks: recall is monotone
+        assert all(a <= b + 1e-15 for a, b in zip(Rs, Rs[1:]))
+        for i, b in enumerate(bws):                                  # each candidate equals the fixed-window ARM
+            wf, ws = orc.windows_of(b, g)
+            _, (rt, rs, _), _ = orc.arm_head(q[0, h], k[0, h], g, PatternParams(wf, ws, 2), orc.SAMPLE_ALG1, 4, 0.9)
+            assert rt == pytest.approx(Rt[i], abs=1e-15) and rs == pytest.approx(Rs[i], abs=1e-15)
+        assert (cls, idx) == orc.decide_plus(Rt, Rs, 0.9)
+        if cls == TEMPORAL:
+            assert window == orc.windows_of(bws[idx], g)[1]
+        elif cls == SPATIAL:
+            assert window == orc.windows_of(bws[idx], g)[0]
+        else:
+            assert window == -1
+    # a bandwidth of 1 keeps everything: recall 1 and Temporal always qualifies
+    cls, idx, window, Rt, Rs = orc.arm_head_plus(q[0, 2], k[0, 2], g, [1.0], 2, orc.SAMPLE_ALG1, 4, 0.9)
+    assert Rt[0] == pytest.approx(1.0) and Rs[0] == pytest.approx(1.0) and cls == TEMPORAL

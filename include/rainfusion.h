@@ -144,6 +144,29 @@ rf_status rf_dense_attn_fwd(const rf_shape *shape, const void *q, const void *k,
                             float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
 
 /*
+ * RainFusion+ (Sec. 4.3, last paragraph): per-head dynamic bandwidth.  ARM evaluates every candidate bandwidth
+ * of the list (ascending, e.g. 0.125, 0.25, 0.5; at most RF_MAX_BANDWIDTHS) on the same approximate scores.
+ * A bandwidth b stands for the windows w_f = floor(b*T), w_s = floor(b*frame_h*frame_w).  A pattern qualifies
+ * if any candidate reaches alpha, Temporal before Spatial as in Algorithm 1, and the head takes the smallest
+ * qualifying bandwidth; otherwise it is Textural.
+ *   bandwidths   host float [n_bandwidths], ascending, each in (0, 1]
+ *   head_window  device int32 [B,H], written: w_s of a Temporal head, w_f of a Spatial head, -1 for Textural
+ *   recall       device float [B,H,2,n_bandwidths] = (Temporal, Spatial) x candidate, written; may be NULL
+ * rf_build_block_mask_plus / rf_sparse_attn_fwd_plus are rf_build_block_mask / rf_sparse_attn_fwd with those
+ * per-head windows in place of params->frame_window / spatial_window (head_window == NULL: identical to them).
+ */
+#define RF_MAX_BANDWIDTHS 4
+rf_status rf_arm_classify_plus(const rf_shape *shape, const rf_params *params, const float *bandwidths,
+                               int32_t n_bandwidths, const void *q, const void *k, int32_t *head_class,
+                               int32_t *head_window, float *recall, void *ws, size_t ws_bytes, void *cuda_stream);
+rf_status rf_build_block_mask_plus(const rf_shape *shape, const rf_params *params, const int32_t *head_class,
+                                   const int32_t *head_window, rf_schedule *out, int32_t *dev_status, void *cuda_stream);
+rf_status rf_sparse_attn_fwd_plus(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
+                                  const void *v, const int32_t *head_class, const int32_t *head_window,
+                                  const rf_schedule *sched, void *o, float *lse, void *ws, size_t ws_bytes,
+                                  int32_t *dev_status, void *cuda_stream);
+
+/*
  * rf_arm_classify for callers that cannot provide a workspace.  (The paper has no counterpart: this is
  * a packaging variant of rf_arm_classify, same kernels, same results.)
  *

@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
            "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
-           "rf_arm_classify_noalloc"]
+           "rf_arm_classify_noalloc", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus"]
 
 
 class rf_shape(C.Structure):
@@ -68,6 +68,12 @@ def load():
     lib.rf_build_block_mask.argtypes = [P(rf_shape), P(rf_params), V, P(rf_schedule), V, V]
     lib.rf_sparse_attn_fwd.restype = I
     lib.rf_sparse_attn_fwd.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
+    lib.rf_arm_classify_plus.restype = I
+    lib.rf_arm_classify_plus.argtypes = [P(rf_shape), P(rf_params), P(C.c_float), C.c_int32, V, V, V, V, V, V, Z, V]
+    lib.rf_build_block_mask_plus.restype = I
+    lib.rf_build_block_mask_plus.argtypes = [P(rf_shape), P(rf_params), V, V, P(rf_schedule), V, V]
+    lib.rf_sparse_attn_fwd_plus.restype = I
+    lib.rf_sparse_attn_fwd_plus.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
     lib.rf_reorder_tokens.restype = I
     lib.rf_reorder_tokens.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, Z, V]
     lib.rf_dense_attn_fwd.restype = I
@@ -169,6 +175,25 @@ def rf_sparse_attn_fwd(shape, params, q, k, v, head_class, sched: Schedule, o, l
     _check(load().rf_sparse_attn_fwd(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), v.data_ptr(),
                                      head_class.data_ptr(), C.byref(sched.c), o.data_ptr(), _ptr(lse), ws.data_ptr(),
                                      ws.numel(), _ptr(dev_status), _stream()), "rf_sparse_attn_fwd")
+
+
+def rf_arm_classify_plus(shape, params, bandwidths, q, k, head_class, head_window, recall, ws):
+    arr = (C.c_float * len(bandwidths))(*bandwidths)
+    _check(load().rf_arm_classify_plus(C.byref(shape), C.byref(params), arr, len(bandwidths), q.data_ptr(), k.data_ptr(),
+                                       head_class.data_ptr(), head_window.data_ptr(), _ptr(recall), ws.data_ptr(),
+                                       ws.numel(), _stream()), "rf_arm_classify_plus")
+
+
+def rf_build_block_mask_plus(shape, params, head_class, head_window, sched: Schedule, dev_status=None):
+    _check(load().rf_build_block_mask_plus(C.byref(shape), C.byref(params), head_class.data_ptr(), _ptr(head_window),
+                                           C.byref(sched.c), _ptr(dev_status), _stream()), "rf_build_block_mask_plus")
+
+
+def rf_sparse_attn_fwd_plus(shape, params, q, k, v, head_class, head_window, sched: Schedule, o, lse, ws, dev_status=None):
+    _check(load().rf_sparse_attn_fwd_plus(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                          head_class.data_ptr(), _ptr(head_window), C.byref(sched.c), o.data_ptr(),
+                                          _ptr(lse), ws.data_ptr(), ws.numel(), _ptr(dev_status), _stream()),
+           "rf_sparse_attn_fwd_plus")
 
 
 def rf_reorder_tokens(shape, params, q, k, v, head_class, ws):

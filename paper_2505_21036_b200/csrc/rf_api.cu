@@ -145,7 +145,7 @@ rf_status rf_schedule_dims(const rf_shape* shape, const rf_params* params, int32
 size_t rf_workspace_bytes(const rf_shape* shape, const rf_params* params) {
   if (check_shape(shape) != RF_OK || check_params(params) != RF_OK) return 0;
   const RfGeom g = make_geom(shape, params);
-  return 3 * tensor_bytes(g) + align_up(rf_arm_scratch_floats(g, params->sample_stride) * sizeof(float));
+  return 3 * tensor_bytes(g) + align_up(rf_arm_scratch_floats(g, params->sample_stride, RF_MAX_BANDWIDTHS) * sizeof(float));
 }
 
 rf_status rf_arm_classify(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
@@ -160,14 +160,46 @@ rf_status rf_arm_classify(const rf_shape* shape, const rf_params* params, const 
   if (ws_bytes < rf_workspace_bytes(shape, params)) return RF_ERR_WORKSPACE_TOO_SMALL;
   const RfGeom g = make_geom(shape, params);
   float* scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + 3 * tensor_bytes(g));
-  cudaError_t e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha,
+  cudaError_t e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, 1, &g.ws, &g.wf,
                                 static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), head_class,
-                                recall, scratch, static_cast<cudaStream_t>(cuda_stream));
+                                nullptr, recall, nullptr, scratch, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
+}
+
+rf_status rf_arm_classify_plus(const rf_shape* shape, const rf_params* params, const float* bandwidths,
+                               int32_t n_bandwidths, const void* q, const void* k, int32_t* head_class,
+                               int32_t* head_window, float* recall, void* ws, size_t ws_bytes, void* cuda_stream) {
+  rf_status st = check_shape(shape);
+  if (st != RF_OK) return st;
+  st = check_params(params);
+  if (st != RF_OK) return st;
+  if (shape->D != 64 && shape->D != 96 && shape->D != 128) return RF_ERR_UNSUPPORTED;
+  if (bandwidths == nullptr || n_bandwidths < 1 || n_bandwidths > RF_MAX_BANDWIDTHS) return RF_ERR_INVALID_ARG;
+  if (q == nullptr || k == nullptr || head_class == nullptr || head_window == nullptr || ws == nullptr) return RF_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return RF_ERR_INVALID_ARG;
+  if (ws_bytes < rf_workspace_bytes(shape, params)) return RF_ERR_WORKSPACE_TOO_SMALL;
+  const RfGeom g = make_geom(shape, params);
+  int ws_list[RF_MAX_BANDWIDTHS], wf_list[RF_MAX_BANDWIDTHS];
+  for (int i = 0; i < n_bandwidths; ++i) {
+    const float b = bandwidths[i];
+    if (!(b > 0.f && b <= 1.f) || (i > 0 && b <= bandwidths[i - 1])) return RF_ERR_INVALID_ARG;
+    wf_list[i] = (int)floor((double)b * g.T);
+    ws_list[i] = (int)floor((double)b * g.S);
+  }
+  float* scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + 3 * tensor_bytes(g));
+  cudaError_t e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, n_bandwidths, ws_list,
+                                wf_list, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+                                head_class, head_window, nullptr, recall, scratch, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }
 
 rf_status rf_build_block_mask(const rf_shape* shape, const rf_params* params, const int32_t* head_class,
                               rf_schedule* out, int32_t* dev_status, void* cuda_stream) {
+  return rf_build_block_mask_plus(shape, params, head_class, nullptr, out, dev_status, cuda_stream);
+}
+
+rf_status rf_build_block_mask_plus(const rf_shape* shape, const rf_params* params, const int32_t* head_class,
+                                   const int32_t* head_window, rf_schedule* out, int32_t* dev_status, void* cuda_stream) {
   rf_status st = check_shape(shape);
   if (st != RF_OK) return st;
   st = check_params(params);
@@ -176,14 +208,22 @@ rf_status rf_build_block_mask(const rf_shape* shape, const rf_params* params, co
     return RF_ERR_INVALID_ARG;
   const RfGeom g = make_geom(shape, params);
   if (out->nQ != g.nQ || out->nKmax != g.nKmax) return RF_ERR_INVALID_ARG;
-  cudaError_t e = rf_launch_build_tiles(g, head_class, out->count, out->kv_tile, out->bitmap, out->kv_len, dev_status,
-                                        static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = rf_launch_build_tiles(g, head_class, head_window, out->count, out->kv_tile, out->bitmap, out->kv_len,
+                                        dev_status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }
 
 rf_status rf_sparse_attn_fwd(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
                              const void* v, const int32_t* head_class, const rf_schedule* sched, void* o, float* lse,
                              void* ws, size_t ws_bytes, int32_t* dev_status, void* cuda_stream) {
+  return rf_sparse_attn_fwd_plus(shape, params, q, k, v, head_class, nullptr, sched, o, lse, ws, ws_bytes, dev_status,
+                                 cuda_stream);
+}
+
+rf_status rf_sparse_attn_fwd_plus(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
+                                  const void* v, const int32_t* head_class, const int32_t* head_window,
+                                  const rf_schedule* sched, void* o, float* lse, void* ws, size_t ws_bytes,
+                                  int32_t* dev_status, void* cuda_stream) {
   rf_status st = check_attn_shape(shape);
   if (st != RF_OK) return st;
   st = check_params(params);
@@ -220,6 +260,7 @@ rf_status rf_sparse_attn_fwd(const rf_shape* shape, const rf_params* params, con
   RfAttnArgs a;
   a.g = g;
   a.head_class = head_class;
+  a.head_window = head_window;
   a.count = sched->count;
   a.kv_tile = sched->kv_tile;
   a.o = static_cast<__nv_bfloat16*>(o);
@@ -267,6 +308,7 @@ rf_status rf_dense_attn_fwd(const rf_shape* shape, const void* q, const void* k,
   RfAttnArgs a;
   a.g = g;
   a.head_class = nullptr;
+  a.head_window = nullptr;
   a.count = nullptr;
   a.kv_tile = nullptr;
   a.o = static_cast<__nv_bfloat16*>(o);

@@ -30,14 +30,17 @@ constexpr int ARM_TMA_WARP = 8, ARM_MMA_WARP = 9;
 
 struct ArmMaps { CUtensorMap q[2], k[2]; };   // per sample: 0 = stride sample, 1 = first-frame sample
 
+constexpr int ARM_MAX_NB = RF_MAX_BANDWIDTHS;   // candidate windows per pattern (1 for plain Algorithm 1)
+
 struct ArmSample {
   int n;          // sampled tokens
   int stride;     // token index of sample m is m * stride
   int pairs;      // CTAs per head: ceil(ceil(n/128) / 2)
-  int want_t;     // accumulate the Temporal mass on this sample
-  int want_s;     // accumulate the Spatial mass on this sample
-  float* out;     // [B*H][3][n_pad]
+  int want_t;     // accumulate the Temporal masses on this sample
+  int want_s;     // accumulate the Spatial masses on this sample
+  float* out;     // [B*H][2*NB+1][n_pad]: Temporal per window, Spatial per window, Textural
 };
+struct ArmWindows { int ws[ARM_MAX_NB], wf[ARM_MAX_NB]; };   // candidate spatial (Temporal) / frame (Spatial) windows
 
 template <int D>
 struct ArmCfg {
@@ -77,10 +80,11 @@ __device__ __forceinline__ void interval_bits(uint32_t (&w)[4], int u0, int a, i
   }
 }
 
-template <int D, bool TEX>
+template <int D, int NB, bool TEX>
 __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_constant__ ArmMaps maps, const RfGeom g,
-                                                                const ArmSample sm0, const ArmSample sm1, int n_pad,
-                                                                float scale_log2, int32_t* dev_status) {
+                                                                const ArmSample sm0, const ArmSample sm1,
+                                                                const ArmWindows win, int n_pad, float scale_log2,
+                                                                int32_t* dev_status) {
   using C = ArmCfg<D>;
   constexpr uint32_t IDESC_S = idesc_bf16(128, 128, 0);
   extern __shared__ uint8_t smem_raw[];
@@ -103,7 +107,6 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
   const bool stream1 = qt0 + 1 < nt;
   const CUtensorMap* map_q = &maps.q[which];
   const CUtensorMap* map_k = &maps.k[which];
-  const bool t_band = sm.want_t && stride == 1;       // positions = sample indices: the Temporal mask is one interval
   const bool t_generic = sm.want_t && stride != 1;    // needs per-key positions
 
   if (tid == 0) {
@@ -175,14 +178,24 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
       const int mc = min(m, n - 1);
       const int tok = mc * stride;
       const int rf = tok / g.S, rp = tok - rf * g.S;
-      // kept key intervals of this row, in sample-index space
-      const int t_lo = rp - g.ws, t_hi = rp + g.ws + 1;                               // first-frame sample only
-      const int s_lo = rf_cdiv(max(rf - g.wf, 0) * g.S, stride);
-      const int s_hi = rf_cdiv((rf + g.wf + 1) * g.S, stride);                         // exclusive
+      // Masks k = 0..NB-1: Temporal with window win.ws[k]; k = NB..2NB-1: Spatial with win.wf[k-NB];
+      // k = 2NB: Textural.  Band masks keep one key interval [lo, hi) per row in sample-index space.
+      constexpr int NM = 2 * NB + 1;
+      int lo[2 * NB], hi[2 * NB];
+#pragma unroll
+      for (int i = 0; i < NB; ++i) {
+        lo[i] = rp - win.ws[i];                                     // first-frame sample: position = index
+        hi[i] = rp + win.ws[i] + 1;
+        lo[NB + i] = rf_cdiv(max(rf - win.wf[i], 0) * g.S, stride);  // stride sample: frames grow with the index
+        hi[NB + i] = rf_cdiv((rf + win.wf[i] + 1) * g.S, stride);
+      }
       const uint32_t t_s = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + j * 256;
       int* attr_p = reinterpret_cast<int*>(base_ptr + C::ATTR) + warp * 256;           // per-warp tables
       int* attr_c = attr_p + 128;
-      float mx = -INFINITY, l_all = 0.f, l_t = 0.f, l_s = 0.f, l_c = 0.f;
+      float mx = -INFINITY, l_all = 0.f;
+      float l_m[NM];
+#pragma unroll
+      for (int k = 0; k < NM; ++k) l_m[k] = 0.f;
 
       for (int u = 0; u < nt; ++u) {
         const int b = u & 1, u0 = u * ARM_TILE;
@@ -217,83 +230,107 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
         }
         const float m_new = fmaxf(mx, fmaxf(m0, m1) * scale_log2);   // finite: every tile holds a real key
         const float corr = ex2f(mx - m_new);
-        l_all *= corr; l_t *= corr; l_s *= corr; l_c *= corr;
+        l_all *= corr;
+#pragma unroll
+        for (int k = 0; k < NM; ++k) l_m[k] *= corr;
         mx = m_new;
 
-        // where does this tile lie relative to the row's kept intervals?  0 outside, 2 inside, 1 crossing
-        const int u1 = min(u0 + ARM_TILE, n);
-        int t_cls = 0, s_cls = 0;
-        if (t_band) {
-          const bool in = t_lo <= u0 && u1 <= t_hi, out = u1 <= t_lo || t_hi <= u0;
-          t_cls = __all_sync(0xffffffffu, in) ? 2 : (__all_sync(0xffffffffu, out) ? 0 : 1);
-        } else if (t_generic) {
-          t_cls = 1;
-        }
-        if (sm.want_s) {
-          const bool in = s_lo <= u0 && u1 <= s_hi, out = u1 <= s_lo || s_hi <= u0;
-          s_cls = __all_sync(0xffffffffu, in) ? 2 : (__all_sync(0xffffffffu, out) ? 0 : 1);
-        }
+        // exponentials once, in place; their sum serves every mask the tile lies wholly inside
         const float2 sc2 = make_float2(scale_log2, scale_log2), mneg = make_float2(-m_new, -m_new);
-        if (!TEX && t_cls != 1 && s_cls != 1) {
-          float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+        float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int c = 0; c < 128; c += 4) {
-            float2 e0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, mneg);
-            float2 e1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, mneg);
-            e0.x = ex2f(e0.x); e0.y = ex2f(e0.y);
-            e1.x = ex2f(e1.x); e1.y = ex2f(e1.y);
-            la = __fadd2_rn(la, e0);
-            lb = __fadd2_rn(lb, e1);
+        for (int c = 0; c < 128; c += 4) {
+          float2 e0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, mneg);
+          float2 e1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, mneg);
+          e0.x = ex2f(e0.x); e0.y = ex2f(e0.y);
+          e1.x = ex2f(e1.x); e1.y = ex2f(e1.y);
+          la = __fadd2_rn(la, e0);
+          lb = __fadd2_rn(lb, e1);
+          s[c] = __float_as_uint(e0.x); s[c + 1] = __float_as_uint(e0.y);
+          s[c + 2] = __float_as_uint(e1.x); s[c + 3] = __float_as_uint(e1.y);
+        }
+        const float bs = (la.x + la.y) + (lb.x + lb.y);
+        l_all += bs;
+
+        // per mask: the tile lies inside the row's kept interval for the whole warp (add the tile sum),
+        // outside it (nothing), or an edge crosses it (masked sum with a 128-bit keep word)
+        const int u1 = min(u0 + ARM_TILE, n);
+        bool table_ready = false;
+#pragma unroll 1
+        for (int k = 0; k < NM; ++k) {
+          const bool is_t = k < NB, is_x = k == 2 * NB;
+          if (is_x ? !TEX : (is_t ? !sm.want_t : !sm.want_s)) continue;
+          const bool by_table = is_x || (is_t && t_generic);
+          int cls = 1;
+          int klo = 0, khi = 0;
+          if (!by_table) {
+#pragma unroll
+            for (int i = 0; i < 2 * NB; ++i)
+              if (i == k) { klo = lo[i]; khi = hi[i]; }
+            const bool in = klo <= u0 && u1 <= khi, out = u1 <= klo || khi <= u0;
+            cls = __all_sync(0xffffffffu, in) ? 2 : (__all_sync(0xffffffffu, out) ? 0 : 1);
           }
-          const float bs = (la.x + la.y) + (lb.x + lb.y);
-          l_all += bs;
-          if (t_cls == 2) l_t += bs;
-          if (s_cls == 2) l_s += bs;
-        } else {
-          // keep words per mask for this row and tile
-          uint32_t wt[4] = {0, 0, 0, 0}, ws[4] = {0, 0, 0, 0}, wx[4] = {0, 0, 0, 0};
-          if (t_band) interval_bits(wt, u0, t_lo, t_hi);
-          if (sm.want_s) interval_bits(ws, u0, s_lo, s_hi);
-          if (TEX || t_generic) {
-            // per-key attributes of the tile, four keys per lane, into this warp's table
-            __syncwarp();
+          float add = 0.f;
+          if (cls == 2) {
+            add = bs;
+          } else if (cls == 1) {
+            uint32_t w[4] = {0, 0, 0, 0};
+            if (!by_table) {
+              interval_bits(w, u0, klo, khi);
+            } else {
+              if (!table_ready) {
+                // per-key attributes of the tile, four keys per lane, into this warp's table
+                __syncwarp();
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int c = lane * 4 + i;
-              const int ktok = min(u0 + c, n - 1) * stride;
-              const int kp = ktok % g.S;
-              const int y = kp / g.Wf, x = kp - y * g.Wf;
-              attr_p[c] = kp;
-              attr_c[c] = (y % g.tau) == (x % g.tau);
+                for (int i = 0; i < 4; ++i) {
+                  const int c = lane * 4 + i;
+                  const int ktok = min(u0 + c, n - 1) * stride;
+                  const int kp = ktok % g.S;
+                  const int y = kp / g.Wf, x = kp - y * g.Wf;
+                  attr_p[c] = kp;
+                  attr_c[c] = (y % g.tau) == (x % g.tau);
+                }
+                __syncwarp();
+                table_ready = true;
+              }
+              int wk = 0;
+#pragma unroll
+              for (int i = 0; i < NB; ++i)
+                if (i == k) wk = win.ws[i];
+#pragma unroll
+              for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t bits = 0;
+#pragma unroll 8
+                for (int c = 0; c < 32; ++c) {
+                  bool keep;
+                  if (is_x) {
+                    keep = attr_c[q4 * 32 + c] != 0;
+                  } else {
+                    const int dp = attr_p[q4 * 32 + c] - rp;
+                    keep = (dp < 0 ? -dp : dp) <= wk;
+                  }
+                  bits |= (keep ? 1u : 0u) << c;
+                }
+                w[q4] = bits;
+              }
             }
-            __syncwarp();
-#pragma unroll 4
-            for (int c = 0; c < 128; ++c) {
-              if (t_generic) { const int dp = attr_p[c] - rp; if ((dp < 0 ? -dp : dp) <= g.ws) wt[c >> 5] |= 1u << (c & 31); }
-              if (TEX && attr_c[c]) wx[c >> 5] |= 1u << (c & 31);
-            }
-          }
-          float bs = 0.f, bt = 0.f, bsp = 0.f, bx = 0.f;
 #pragma unroll
-          for (int c = 0; c < 128; ++c) {
-            const float p = ex2f(fmaf(__uint_as_float(s[c]), scale_log2, -m_new));
-            bs += p;
-            if ((wt[c >> 5] >> (c & 31)) & 1u) bt += p;
-            if ((ws[c >> 5] >> (c & 31)) & 1u) bsp += p;
-            if (TEX) { if ((wx[c >> 5] >> (c & 31)) & 1u) bx += p; }
+            for (int c = 0; c < 128; ++c)
+              if ((w[c >> 5] >> (c & 31)) & 1u) add += __uint_as_float(s[c]);
           }
-          l_all += bs;
-          l_t += bt;
-          l_s += bsp;
-          l_c += bx;
+#pragma unroll
+          for (int i = 0; i < NM; ++i)
+            if (i == k) l_m[i] += add;
         }
       }
       if (m < n) {
-        float* out = sm.out + (size_t)bh * 3 * n_pad;
+        float* out = sm.out + (size_t)bh * NM * n_pad;
         const float inv = 1.f / l_all;
-        if (sm.want_t) out[m] = l_t * inv;
-        if (sm.want_s) out[n_pad + m] = l_s * inv;
-        if (TEX) out[2 * n_pad + m] = l_c * inv;
+#pragma unroll
+        for (int k = 0; k < NM; ++k) {
+          const bool is_t = k < NB, is_x = k == 2 * NB;
+          if (is_x ? TEX : (is_t ? sm.want_t != 0 : sm.want_s != 0)) out[(size_t)k * n_pad + m] = l_m[k] * inv;
+        }
       }
     }
   }
@@ -307,64 +344,87 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
   }
 }
 
-// One CTA per head: mean of the per-row recalls in a fixed order, then Algorithm 1.
-__global__ void __launch_bounds__(256) rf_arm_decide_kernel(int n_loc, int n_glb, int n_pad, int sample_mode, float alpha,
+// One CTA per head: means of the per-row recalls in a fixed order, then the decision.
+//   plain (head_window == nullptr, nb = 1): Algorithm 1.
+//   dynamic bandwidth: a pattern qualifies if any candidate window reaches alpha, Temporal before Spatial;
+//   the head takes the smallest qualifying window (candidates ascend); Textural heads get window -1.
+__global__ void __launch_bounds__(256) rf_arm_decide_kernel(int nb, int nb_user, int n_loc, int n_glb, int n_pad, int sample_mode,
+                                                             float alpha, ArmWindows win, int with_tex,
                                                              const float* __restrict__ rows_loc,
                                                              const float* __restrict__ rows_glb,
-                                                             int32_t* __restrict__ head_class, float* __restrict__ recall) {
-  __shared__ double red[3][256];
+                                                             int32_t* __restrict__ head_class,
+                                                             int32_t* __restrict__ head_window, float* __restrict__ recall,
+                                                             float* __restrict__ recall_plus) {
+  __shared__ double red[2 * ARM_MAX_NB + 1][256];
   const int bh = blockIdx.x, tid = threadIdx.x;
-  const float* gl = rows_glb + (size_t)bh * 3 * n_pad;
-  const float* lo = rows_loc + (size_t)bh * 3 * n_pad;
+  const int nm = 2 * nb + 1;
+  const float* gl = rows_glb + (size_t)bh * nm * n_pad;
+  const float* lo = rows_loc + (size_t)bh * nm * n_pad;
   const bool local_t = sample_mode == RF_SAMPLE_ALG1;
-  const float* src[3] = {local_t ? lo : gl, gl + n_pad, gl + 2 * n_pad};
-  const int cnt[3] = {local_t ? n_loc : n_glb, n_glb, n_glb};
-  const int nw = recall != nullptr ? 3 : 2;   // the Textural recall is only accumulated when recalls are wanted
-  for (int w = 0; w < 3; ++w) {
-    double s = 0.0;
-    if (w < nw)
-      for (int i = tid; i < cnt[w]; i += 256) s += (double)src[w][i];
-    red[w][tid] = s;
+  for (int k = 0; k < nm; ++k) {
+    const bool is_t = k < nb, is_x = k == 2 * nb;
+    const float* src = ((is_t && local_t) ? lo : gl) + (size_t)k * n_pad;
+    const int cnt = (is_t && local_t) ? n_loc : n_glb;
+    double acc = 0.0;
+    if (!is_x || with_tex)
+      for (int i = tid; i < cnt; i += 256) acc += (double)src[i];
+    red[k][tid] = acc;
   }
   __syncthreads();
   for (int o = 128; o > 0; o >>= 1) {
     if (tid < o)
-      for (int w = 0; w < 3; ++w) red[w][tid] += red[w][tid + o];
+      for (int k = 0; k < nm; ++k) red[k][tid] += red[k][tid + o];
     __syncthreads();
   }
   if (tid == 0) {
-    const float Rt = (float)(red[0][0] / cnt[0]), Rs = (float)(red[1][0] / cnt[1]), Rc = (float)(red[2][0] / cnt[2]);
-    if (recall) { recall[bh * 3] = Rt; recall[bh * 3 + 1] = Rs; recall[bh * 3 + 2] = Rc; }
-    head_class[bh] = Rt >= alpha ? RF_TEMPORAL : (Rs >= alpha ? RF_SPATIAL : RF_TEXTURAL);
+    float R[2 * ARM_MAX_NB + 1];
+    for (int k = 0; k < nm; ++k) R[k] = (float)(red[k][0] / ((k < nb && local_t) ? n_loc : n_glb));
+    if (head_window == nullptr) {
+      const float Rt = R[0], Rs = R[nb], Rc = R[2 * nb];
+      if (recall) { recall[bh * 3] = Rt; recall[bh * 3 + 1] = Rs; recall[bh * 3 + 2] = Rc; }
+      head_class[bh] = Rt >= alpha ? RF_TEMPORAL : (Rs >= alpha ? RF_SPATIAL : RF_TEXTURAL);
+    } else {
+      int cls = RF_TEXTURAL, window = -1;
+      // nb slots were evaluated (the caller's nb_user candidates, padded by repeating the last one)
+      for (int i = nb_user - 1; i >= 0; --i)
+        if (R[nb + i] >= alpha) { cls = RF_SPATIAL; window = win.wf[i]; }
+      for (int i = nb_user - 1; i >= 0; --i)
+        if (R[i] >= alpha) { cls = RF_TEMPORAL; window = win.ws[i]; }
+      head_class[bh] = cls;
+      head_window[bh] = window;
+      if (recall_plus)
+        for (int i = 0; i < nb_user; ++i) {
+          recall_plus[(bh * 2) * nb_user + i] = R[i];
+          recall_plus[(bh * 2 + 1) * nb_user + i] = R[nb + i];
+        }
+    }
   }
 }
 
-template <int D, bool TEX>
-cudaError_t launch_arm_t(const ArmMaps& maps, const RfGeom& g, const ArmSample& s0, const ArmSample& s1, int n_pad,
-                         int32_t* dev_status, cudaStream_t st) {
+template <int D, int NB, bool TEX>
+cudaError_t launch_arm_t(const ArmMaps& maps, const RfGeom& g, const ArmSample& s0, const ArmSample& s1,
+                         const ArmWindows& win, int n_pad, int32_t* dev_status, cudaStream_t st) {
   static bool configured[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev >= 0 && dev < 64 && !configured[dev]) {
-    e = cudaFuncSetAttribute(rf_arm_kernel<D, TEX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ArmCfg<D>::ALLOC);
+    e = cudaFuncSetAttribute(rf_arm_kernel<D, NB, TEX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ArmCfg<D>::ALLOC);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   dim3 grid(s0.pairs + s1.pairs, g.B * g.H);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
-  rf_arm_kernel<D, TEX><<<grid, ARM_THREADS, ArmCfg<D>::ALLOC, st>>>(maps, g, s0, s1, n_pad, scale_log2, dev_status);
+  rf_arm_kernel<D, NB, TEX><<<grid, ARM_THREADS, ArmCfg<D>::ALLOC, st>>>(maps, g, s0, s1, win, n_pad, scale_log2, dev_status);
   return cudaGetLastError();
 }
 
-cudaError_t launch_arm_d(bool tex, const ArmMaps& maps, const RfGeom& g, const ArmSample& s0, const ArmSample& s1,
-                         int n_pad, cudaStream_t st) {
-  switch (g.D) {
-    case 64: return tex ? launch_arm_t<64, true>(maps, g, s0, s1, n_pad, nullptr, st) : launch_arm_t<64, false>(maps, g, s0, s1, n_pad, nullptr, st);
-    case 96: return tex ? launch_arm_t<96, true>(maps, g, s0, s1, n_pad, nullptr, st) : launch_arm_t<96, false>(maps, g, s0, s1, n_pad, nullptr, st);
-    case 128: return tex ? launch_arm_t<128, true>(maps, g, s0, s1, n_pad, nullptr, st) : launch_arm_t<128, false>(maps, g, s0, s1, n_pad, nullptr, st);
-  }
-  return cudaErrorInvalidValue;
+template <int D>
+cudaError_t launch_arm_n(bool plus, bool tex, const ArmMaps& maps, const RfGeom& g, const ArmSample& s0,
+                         const ArmSample& s1, const ArmWindows& win, int n_pad, cudaStream_t st) {
+  if (plus) return launch_arm_t<D, ARM_MAX_NB, false>(maps, g, s0, s1, win, n_pad, nullptr, st);
+  return tex ? launch_arm_t<D, 1, true>(maps, g, s0, s1, win, n_pad, nullptr, st)
+             : launch_arm_t<D, 1, false>(maps, g, s0, s1, win, n_pad, nullptr, st);
 }
 
 int arm_n_pad(const RfGeom& g, int omega) {
@@ -375,18 +435,28 @@ int arm_n_pad(const RfGeom& g, int omega) {
 
 }  // namespace
 
-size_t rf_arm_scratch_floats(const RfGeom& g, int omega) { return (size_t)2 * g.B * g.H * 3 * arm_n_pad(g, omega); }
+size_t rf_arm_scratch_floats(const RfGeom& g, int omega, int nb) {
+  return (size_t)2 * g.B * g.H * (2 * nb + 1) * arm_n_pad(g, omega);
+}
 
-cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, const __nv_bfloat16* q,
-                          const __nv_bfloat16* k, int32_t* head_class, float* recall, float* row_scratch,
-                          cudaStream_t st) {
+cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, int nb, const int* ws_list,
+                          const int* wf_list, const __nv_bfloat16* q, const __nv_bfloat16* k, int32_t* head_class,
+                          int32_t* head_window, float* recall, float* recall_plus, float* row_scratch, cudaStream_t st) {
+  const bool plus = head_window != nullptr;
+  const int NB = plus ? ARM_MAX_NB : 1;           // windows the kernel evaluates (candidate list padded by repetition)
+  if (nb < 1 || nb > NB) return cudaErrorInvalidValue;
+  ArmWindows win;
+  for (int i = 0; i < ARM_MAX_NB; ++i) {
+    win.ws[i] = ws_list[i < nb ? i : nb - 1];
+    win.wf[i] = wf_list[i < nb ? i : nb - 1];
+  }
   const int n_pad = arm_n_pad(g, omega);
   const int n_glb = rf_cdiv(g.Nv, omega), n_loc = g.S;
-  float* rows_glb = row_scratch;
-  float* rows_loc = row_scratch + (size_t)g.B * g.H * 3 * n_pad;
-  const bool alg1 = sample_mode == RF_SAMPLE_ALG1;
-  const bool tex = recall != nullptr;   // the Textural recall is a diagnostic: Algorithm 1 does not use it
   const int heads = g.B * g.H;
+  float* rows_glb = row_scratch;
+  float* rows_loc = row_scratch + (size_t)heads * (2 * NB + 1) * n_pad;
+  const bool alg1 = sample_mode == RF_SAMPLE_ALG1;
+  const bool tex = !plus && recall != nullptr;   // the Textural recall is a diagnostic: Algorithm 1 does not use it
   const size_t row_bytes = (size_t)g.D * 2, head_bytes = (size_t)g.N * g.D * 2;
   ArmMaps maps;
   bool ok = rf_encode_rows_map(&maps.q[0], q, g.D, n_glb, row_bytes * omega, head_bytes, heads) &&
@@ -399,10 +469,16 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
   s0.want_t = alg1 ? 0 : 1; s0.want_s = 1; s0.out = rows_glb;
   s1.n = n_loc; s1.stride = 1; s1.pairs = alg1 ? rf_cdiv(rf_cdiv(n_loc, ARM_TILE), 2) : 0;
   s1.want_t = 1; s1.want_s = 0; s1.out = rows_loc;
-  cudaError_t e = launch_arm_d(tex, maps, g, s0, s1, n_pad, st);
+  cudaError_t e;
+  switch (g.D) {
+    case 64: e = launch_arm_n<64>(plus, tex, maps, g, s0, s1, win, n_pad, st); break;
+    case 96: e = launch_arm_n<96>(plus, tex, maps, g, s0, s1, win, n_pad, st); break;
+    case 128: e = launch_arm_n<128>(plus, tex, maps, g, s0, s1, win, n_pad, st); break;
+    default: e = cudaErrorInvalidValue;
+  }
   if (e != cudaSuccess) return e;
-  rf_arm_decide_kernel<<<heads, 256, 0, st>>>(n_loc, n_glb, n_pad, sample_mode, alpha, rows_loc, rows_glb, head_class,
-                                              recall);
+  rf_arm_decide_kernel<<<heads, 256, 0, st>>>(NB, nb, n_loc, n_glb, n_pad, sample_mode, alpha, win, tex ? 1 : 0, rows_loc,
+                                              rows_glb, head_class, head_window, recall, recall_plus);
   return cudaGetLastError();
 }
 
@@ -438,14 +514,15 @@ extern "C" rf_status rf_arm_classify_noalloc(const rf_shape* shape, const rf_par
   if (g.D != 64 && g.D != 96 && g.D != 128) return RF_ERR_UNSUPPORTED;
   if (q == nullptr || k == nullptr || head_class == nullptr) return RF_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(q) & 15u) != 0 || (reinterpret_cast<uintptr_t>(k) & 15u) != 0) return RF_ERR_INVALID_ARG;
-  if (rf_arm_scratch_floats(g, params->sample_stride) > (size_t)RF_ARM_STATIC_SCRATCH_FLOATS)
+  if (rf_arm_scratch_floats(g, params->sample_stride, 1) > (size_t)RF_ARM_STATIC_SCRATCH_FLOATS)
     return RF_ERR_STATIC_SCRATCH_TOO_SMALL;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return RF_ERR_CUDA;
   cudaError_t e;
   float* scratch = static_scratch_ptr(dev, &e);
   if (scratch == nullptr) return RF_ERR_CUDA;
-  e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, static_cast<const __nv_bfloat16*>(q),
-                    static_cast<const __nv_bfloat16*>(k), head_class, recall, scratch, static_cast<cudaStream_t>(cuda_stream));
+  e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, 1, &g.ws, &g.wf,
+                    static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), head_class, nullptr, recall,
+                    nullptr, scratch, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }

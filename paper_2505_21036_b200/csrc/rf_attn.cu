@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + C::MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + C::MISC + 8);
 
-  const RfGeom& g = a.g;
+  RfGeom g = a.g;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = blockIdx.y;
   const int qt0 = 2 * blockIdx.x, qt1 = qt0 + 1;
@@ -186,6 +186,11 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       if (tid == 0) rf_report(a.dev_status, RF_ERR_INVALID_ARG);
       cls = RF_DENSE;
     }
+  }
+  if (a.head_window != nullptr) {   // dynamic bandwidth: this head's own window
+    const int w = a.head_window[bh];
+    if (cls == RF_SPATIAL && w >= 0) g.wf = w;
+    if (cls == RF_TEMPORAL && w >= 0) g.ws = w;
   }
   const bool perm = cls == RF_TEMPORAL && g.permute;
   const bool tex = cls == RF_TEXTURAL;

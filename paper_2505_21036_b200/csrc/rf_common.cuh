@@ -35,15 +35,19 @@ __host__ __device__ __forceinline__ int rf_kv_len(const RfGeom& g, int cls) {
 }
 
 // Launchers implemented in the .cu files (host).
-cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, int32_t* count, int32_t* kv_tile,
-                                  uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st);
+// head_window (nullable): per-head window replacing g.wf (Spatial heads) / g.ws (Temporal heads)
+cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, const int32_t* head_window, int32_t* count,
+                                  int32_t* kv_tile, uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st);
 cudaError_t rf_launch_gather(const RfGeom& g, const int32_t* head_class, const __nv_bfloat16* q,
                              const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* wq, __nv_bfloat16* wk,
                              __nv_bfloat16* wv, cudaStream_t st);
-cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, const __nv_bfloat16* q,
-                          const __nv_bfloat16* k, int32_t* head_class, float* recall, float* row_scratch,
-                          cudaStream_t st);
-size_t rf_arm_scratch_floats(const RfGeom& g, int omega);
+// nb candidate windows per pattern (ws_list for Temporal, wf_list for Spatial, ascending).  head_window == nullptr:
+// plain Algorithm 1 on the first candidate (recall: [B,H,3] or null).  Otherwise dynamic bandwidth: head_window
+// receives each head's chosen window, recall_plus ([B,H,2,nb] or null) the candidates' recalls.
+cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, int nb, const int* ws_list,
+                          const int* wf_list, const __nv_bfloat16* q, const __nv_bfloat16* k, int32_t* head_class,
+                          int32_t* head_window, float* recall, float* recall_plus, float* row_scratch, cudaStream_t st);
+size_t rf_arm_scratch_floats(const RfGeom& g, int omega, int nb);
 // Tensor map over bf16 rows: [heads][rows][D] with the given row and head strides in bytes (multiples of 16),
 // box = 64 columns x 128 rows, 128-byte swizzle, zero fill past `rows`.
 bool rf_encode_rows_map(CUtensorMap* m, const void* ptr, int D, int rows, size_t row_stride_bytes,
@@ -54,6 +58,7 @@ rf_status rf_checked_geom(const rf_shape* shape, const rf_params* params, RfGeom
 struct RfAttnArgs {
   RfGeom g;
   const int32_t* head_class;  // nullptr: every head Dense, implicit full tile list
+  const int32_t* head_window; // nullable: per-head window replacing g.wf (Spatial) / g.ws (Temporal)
   const int32_t* count;
   const int32_t* kv_tile;
   __nv_bfloat16* o;

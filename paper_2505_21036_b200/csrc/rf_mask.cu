@@ -62,6 +62,7 @@ __device__ int tile_flag(const RfGeom& g, int cls, int a, int b) {
 
 // One CTA per (query tile, head): flags for all key tiles, then an ordered compaction.
 __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int32_t* __restrict__ head_class,
+                                                              const int32_t* __restrict__ head_window,
                                                               int32_t* __restrict__ count, int32_t* __restrict__ kv_tile,
                                                               uint32_t* __restrict__ bitmap, int32_t* __restrict__ kv_len,
                                                               int32_t* dev_status) {
@@ -72,6 +73,11 @@ __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int
   if (cls < 0 || cls > 3) {
     if (threadIdx.x == 0) rf_report(dev_status, RF_ERR_INVALID_ARG);
     cls = RF_DENSE;
+  }
+  if (head_window != nullptr) {   // dynamic bandwidth: this head's own window
+    const int w = head_window[bh];
+    if (cls == RF_SPATIAL && w >= 0) g.wf = w;
+    if (cls == RF_TEMPORAL && w >= 0) g.ws = w;
   }
   const int Lkv = rf_kv_len(g, cls);
   const int nK = rf_cdiv(Lkv, g.BN);
@@ -156,10 +162,10 @@ __global__ void __launch_bounds__(256) rf_gather_kernel(RfGeom g, const int32_t*
 
 }  // namespace
 
-cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, int32_t* count, int32_t* kv_tile,
-                                  uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st) {
+cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, const int32_t* head_window, int32_t* count,
+                                  int32_t* kv_tile, uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st) {
   dim3 grid(g.nQ, g.B * g.H);
-  rf_build_tiles_kernel<<<grid, 256, 0, st>>>(g, head_class, count, kv_tile, bitmap, kv_len, dev_status);
+  rf_build_tiles_kernel<<<grid, 256, 0, st>>>(g, head_class, head_window, count, kv_tile, bitmap, kv_len, dev_status);
   return cudaGetLastError();
 }
 

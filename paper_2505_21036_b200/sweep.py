@@ -51,13 +51,57 @@ def run_case(wl, classes, permute, q, k, v, o, status, reps):
     return ms, listed, partial, sched.nQ * sched.nKmax * wl.B * wl.H
 
 
+def run_plus(name, bandwidths, reps):
+    """Dynamic bandwidth (RainFusion+) on the seeded planted inputs of a workload: ARM picks a window per head."""
+    import numpy as np
+    wl = synth.WORKLOADS[name]
+    q, k, v = (torch.from_numpy(x.view(np.int16)).cuda().view(torch.bfloat16) for x in synth.make_qkv(wl))
+    o = torch.empty_like(q)
+    shape, params = api.shape_of(wl), api.params_of(wl)
+    ws = api.alloc_workspace(shape, params, "cuda")
+    sched = api.Schedule(shape, params, "cuda")
+    hc = torch.zeros((wl.B, wl.H), dtype=torch.int32, device="cuda")
+    hw = torch.zeros((wl.B, wl.H), dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+    arm_ms = timed(lambda: api.rf_arm_classify_plus(shape, params, bandwidths, q, k, hc, hw, None, ws))
+    api.rf_build_block_mask_plus(shape, params, hc, hw, sched, status)
+    attn_ms = timed(lambda: api.rf_sparse_attn_fwd_plus(shape, params, q, k, v, hc, hw, sched, o, None, ws, status))
+    listed = int(sched.count.sum().item())
+    tf = 4.0 * 128 * 128 * wl.D * listed / (attn_ms * 1e-3) / 1e12
+    assert int(status.item()) == 0
+    picks = sorted(zip(hc.cpu().numpy().reshape(-1).tolist(), hw.cpu().numpy().reshape(-1).tolist()))
+    hist = {}
+    for c, w in picks:
+        hist[f"class{c}/window{w}"] = hist.get(f"class{c}/window{w}", 0) + 1
+    print(json.dumps({"workload": name, "variant": "dynamic bandwidth", "bandwidths": bandwidths, "arm_ms": arm_ms,
+                      "attn_ms": attn_ms, "arm_overhead_pct": 100 * arm_ms / attn_ms, "picks": hist,
+                      "tile_density": listed / float(wl.B * wl.H * sched.nQ * sched.nKmax), "computed_tile_tflops": tf,
+                      "dense_equiv_tflops": 4.0 * wl.B * wl.H * wl.N ** 2 * wl.D / (attn_ms * 1e-3) / 1e12}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--shapes", nargs="+", default=["sweep_8x1024", "sweep_16x2040", "sweep_33x3600"])
     ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--plus", metavar="WORKLOAD", help="run the dynamic-bandwidth variant on this workload and exit")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("sweep: needs a CUDA device")
+    if args.plus:
+        run_plus(args.plus, [0.125, 0.25, 0.5], args.reps)
+        return
     peak = measured_peak()
     for name in args.shapes:
         wl = synth.WORKLOADS[name]

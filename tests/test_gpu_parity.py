@@ -206,3 +206,56 @@ def test_boundary_spotlight_and_poison(cls, permute, inside):
     err = np.abs(O[0, 0] - Or)
     assert err.max() <= 5e-2 * max(1.0, np.abs(Or).max()), err.max()
     assert np.abs(lse[0, 0] - lr).max() <= 5e-3
+
+
+# ------------------------------------------------------------------ degenerate shapes and parameters
+
+@pytest.mark.parametrize("kw", [
+    dict(T=1, fh=9, fw=10, L=5),            # a single frame
+    dict(T=5, fh=6, fw=7, L=0),             # no text tokens
+    dict(T=3, fh=16, fw=8, L=0),            # N = 384: exactly three tiles, no ragged tail
+    dict(T=4, fh=5, fw=5, L=3, wf=0, ws=0), # windows of zero
+    dict(T=4, fh=5, fw=5, L=3, wf=9, ws=99),# windows wider than the extents: dense masks
+    dict(T=4, fh=5, fw=6, L=2, tau=1),      # stride 1: the checkerboard keeps everything
+    dict(T=3, fh=3, fw=5, L=2, tau=4),      # stride not dividing the frame
+])
+def test_edge_shapes_all_patterns(kw):
+    wl = synth.small_workload("edge_shape", H=4, D=64, B=2, **kw)
+    for permute in (1, 0):
+        run = gu.Run(wl, temporal_permute=permute)
+        classes = [S_, T_, X_, D_]
+        run.force_classes(classes * wl.B)
+        run.build()
+        O, lse = run.sparse()
+        g, pp = gu.geom(wl), gu.pparams(wl)
+        for b in range(wl.B):
+            for h, cls in enumerate(classes):
+                ref = gu.oracle_lists(wl, cls, 128, permute)
+                assert run.lists(b, h) == [ref[a] for a in range(run.sched.nQ)]
+                Or, lr = orc.masked_attention(run.q_bits[b, h], run.k_bits[b, h], run.v_bits[b, h], cls, g, pp)
+                gu.check_attention(O[b, h], lse[b, h], Or, lr, f"{kw} b={b} class {cls} permute={permute}", strict=False)
+
+
+def test_arm_edge_shapes():
+    for kw in (dict(T=1, fh=9, fw=10, L=5, omega=1), dict(T=5, fh=6, fw=7, L=0, omega=3), dict(T=2, fh=20, fw=20, L=4, omega=7)):
+        for mode in (0, 1):
+            wl = synth.small_workload("arm_edge", H=3, D=64, B=2, mode=mode, wf=1, ws=5, **kw)
+            check_arm(wl)
+
+
+def test_scores_with_large_dynamic_range_do_not_overflow():
+    """Logits that jump by far more than the lazy-rescale threshold between tiles, and rows whose first
+    tiles are fully masked: the running maximum must be raised (and O rescaled) exactly."""
+    wl = synth.small_workload("range", H=2, D=64, T=6, fh=12, fw=11, L=37, wf=1, ws=20)
+    q, k, v = synth.make_head(wl, 0, 0, kind="none")
+    qf, kf = synth.bf16_bits_to_f32(q).copy(), synth.bf16_bits_to_f32(k).copy()
+    qf[:, 0] = 8.0
+    kf[:, 0] = np.linspace(-40.0, 40.0, wl.N)          # logits grow steadily along the key axis: every tile raises
+    qb, kb = synth.f32_to_bf16_bits(qf), synth.f32_to_bf16_bits(kf)
+    run = gu.Run(wl, qkv=(np.stack([qb, qb])[None], np.stack([kb, kb])[None], np.stack([v, v])[None]))
+    run.force_classes([D_, S_])
+    run.build()
+    O, lse = run.sparse()
+    for h, cls in enumerate([D_, S_]):
+        Or, lr = orc.masked_attention(qb, kb, v, cls, gu.geom(wl), gu.pparams(wl))
+        gu.check_attention(O[0, h], lse[0, h], Or, lr, f"range class {cls}", strict=False)

@@ -279,7 +279,7 @@ def run_cuda(args, wl):
             "clocks": clocks,
             "e2e": {"value": dist_util.replica_throughput(dflops, e2e_ms, world) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 3 * q.numel() * 2, "d2h_bytes_per_step": o.numel() * 2},
-            "gpu_launches": args.steps * (6 if wl.sample_mode == 0 else 5),
+            "gpu_launches": args.steps * 5,   # rf_arm_kernel, rf_arm_decide_kernel, rf_build_tiles_kernel, rf_gather_kernel, rf_attn_kernel
             "breakdown_ms": {"arm": arm_ms, "block_mask": mask_ms, "sparse_attn_call": sparse_ms, "reorder": reorder_ms,
                              "attn_kernel": attn_kernel_ms, "dense_attn_call": dense_ms},
             "arm_overhead_pct": 100.0 * arm_ms / sparse_ms,

@@ -45,7 +45,7 @@ struct ArmWindows { int ws[ARM_MAX_NB], wf[ARM_MAX_NB]; };   // candidate spatia
 template <int D>
 struct ArmCfg {
   static constexpr int KB = (D + 63) / 64;
-  static constexpr int COL1 = D - 64;
+  static constexpr int COL1 = 64;   // D = 96: the second 64-column box reaches past the tensor and is zero-filled
   static constexpr uint32_t BLK = 128 * 128;
   static constexpr uint32_t TILE = KB * BLK;
   static constexpr int NK = D == 64 ? 6 : 4;
@@ -59,7 +59,7 @@ struct ArmCfg {
   static constexpr uint32_t ALLOC = TOTAL + 1024;
   static_assert(ALLOC <= 227 * 1024, "exceeds the shared memory a CTA can opt in to");
   static __host__ __device__ constexpr uint32_t koff(int ks) {
-    return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks * 16 - COL1) * 2u;
+    return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks - 4) * 32u;
   }
 };
 

@@ -30,15 +30,17 @@ struct Maps { CUtensorMap m[8]; };
 template <int D>
 struct Cfg {
   static constexpr int KB = (D + 63) / 64;            // 64-column (128-byte) blocks per row
-  // first column of block kb: D = 96 is held as two overlapping 64-column blocks, [0,64) and [32,96)
-  static constexpr int COL1 = D - 64;
+  // first column of the second block.  D = 96 is fetched as columns [0,64) and [64,128): the TMA box
+  // reaches past the tensor's 96 columns and the missing ones arrive as zeros, so that P V can run as
+  // one N = 128 MMA per k-step (the 32 extra accumulator columns stay zero and are never stored)
+  static constexpr int COL1 = 64;
   static constexpr uint32_t BLK = 128 * 128;          // bytes of one 128-row x 64-col bf16 block
   static constexpr uint32_t TILE = KB * BLK;          // bytes of one 128-row tile
   static constexpr int NK = D == 64 ? 4 : 2;          // K ring depth
   static constexpr int NV = D == 64 ? 4 : 3;          // V ring depth
   // byte offset, inside a tile, of the 16 columns of k-step ks of the Q K^T contraction
   static __host__ __device__ constexpr uint32_t koff(int ks) {
-    return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks * 16 - COL1) * 2u;
+    return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks - 4) * 32u;
   }
   static constexpr uint32_t Q = 0;
   static constexpr uint32_t K0 = Q + 2 * TILE;
@@ -164,8 +166,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   using C = Cfg<D>;
   constexpr int KB = C::KB;
   constexpr uint32_t IDESC_S = idesc_bf16(BM, BN, 0);
-  constexpr uint32_t IDESC_PV = idesc_bf16(BM, D == 96 ? 64 : D, 1);
-  constexpr uint32_t IDESC_PV32 = idesc_bf16(BM, 32, 1);   // D = 96: columns [64, 96) of O
+  constexpr uint32_t IDESC_PV = idesc_bf16(BM, D == 96 ? 128 : D, 1);
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -288,8 +289,6 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
 #pragma unroll
         for (int k = 0; k < BN / 16; ++k) {
           mma_ts(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
-          if (D == 96)  // columns [64, 96): the upper half of the second block's 128-byte rows
-            mma_ts(t_o + 64, t_p + k * 8, desc(b0 + ((C::BLK + k * 2048 + 64) >> 4)), IDESC_PV32, (!first) || k > 0);
         }
         tc_commit(bar(C::B_OF + j));
       };

@@ -139,6 +139,16 @@ rf_status rf_sparse_attn_fwd(const rf_shape *shape, const rf_params *params, con
 rf_status rf_reorder_tokens(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
                             const void *v, const int32_t *head_class, void *ws, size_t ws_bytes, void *cuda_stream);
 
+/*
+ * Self-test of the device-side failure handling (no counterpart in the paper).  Every wait inside the kernels
+ * (on TMA data, on the tensor cores, on another warp role) is bounded; when one runs out the CTA stops waiting,
+ * reports RF_ERR_TIMEOUT through dev_status and still terminates normally.  This entry point launches one warp
+ * that waits limit_ms (1..1000) on a barrier nobody arrives at, so that the mechanism can be exercised without
+ * faulting or hanging the GPU.  On return (after the stream is synchronised) *dev_status is RF_ERR_TIMEOUT if it
+ * was 0 before, and *waits_returned is 4: neither wait succeeded, the abort flag is set.
+ */
+rf_status rf_selftest_wait_timeout(int32_t *dev_status, int32_t limit_ms, int32_t *waits_returned, void *cuda_stream);
+
 /* Full 3D attention (Eq. 1-2, all-zero mask): the same kernel walking every tile.  ws may be NULL. */
 rf_status rf_dense_attn_fwd(const rf_shape *shape, const void *q, const void *k, const void *v, void *o,
                             float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);

@@ -19,7 +19,7 @@ _lib = None
 
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
            "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
-           "rf_arm_classify_noalloc", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus"]
+           "rf_arm_classify_noalloc", "rf_selftest_wait_timeout", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus"]
 
 
 class rf_shape(C.Structure):
@@ -74,6 +74,8 @@ def load():
     lib.rf_build_block_mask_plus.argtypes = [P(rf_shape), P(rf_params), V, V, P(rf_schedule), V, V]
     lib.rf_sparse_attn_fwd_plus.restype = I
     lib.rf_sparse_attn_fwd_plus.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
+    lib.rf_selftest_wait_timeout.restype = I
+    lib.rf_selftest_wait_timeout.argtypes = [V, C.c_int32, V, V]
     lib.rf_reorder_tokens.restype = I
     lib.rf_reorder_tokens.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, Z, V]
     lib.rf_dense_attn_fwd.restype = I
@@ -194,6 +196,11 @@ def rf_sparse_attn_fwd_plus(shape, params, q, k, v, head_class, head_window, sch
                                           head_class.data_ptr(), _ptr(head_window), C.byref(sched.c), o.data_ptr(),
                                           _ptr(lse), ws.data_ptr(), ws.numel(), _ptr(dev_status), _stream()),
            "rf_sparse_attn_fwd_plus")
+
+
+def rf_selftest_wait_timeout(dev_status, limit_ms, waits_returned):
+    _check(load().rf_selftest_wait_timeout(dev_status.data_ptr(), limit_ms, waits_returned.data_ptr(), _stream()),
+           "rf_selftest_wait_timeout")
 
 
 def rf_reorder_tokens(shape, params, q, k, v, head_class, ws):

@@ -270,6 +270,12 @@ rf_status rf_sparse_attn_fwd_plus(const rf_shape* shape, const rf_params* params
   return rf_launch_attention(a, maps, stream);
 }
 
+rf_status rf_selftest_wait_timeout(int32_t* dev_status, int32_t limit_ms, int32_t* waits_returned, void* cuda_stream) {
+  if (dev_status == nullptr || waits_returned == nullptr || limit_ms < 1 || limit_ms > 1000) return RF_ERR_INVALID_ARG;
+  return rf_launch_selftest_timeout(dev_status, (uint64_t)limit_ms * 1000000ull, waits_returned,
+                                    static_cast<cudaStream_t>(cuda_stream));
+}
+
 rf_status rf_reorder_tokens(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
                             const void* v, const int32_t* head_class, void* ws, size_t ws_bytes, void* cuda_stream) {
   rf_status st = check_shape(shape);

@@ -491,6 +491,30 @@ rf_status launch(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st) 
 
 }  // namespace
 
+// Self-test of the bounded-wait machinery every kernel here relies on: one warp waits on an mbarrier that
+// nothing ever arrives at.  The wait must give up after limit_ns, raise the CTA's abort flag, report
+// RF_ERR_TIMEOUT to *dev_status, let a second wait return at once, and the kernel must exit normally.
+__global__ void rf_selftest_timeout_kernel(int32_t* dev_status, uint64_t limit_ns, int32_t* waits_returned) {
+  __shared__ __align__(8) uint64_t barrier;
+  __shared__ int abort_flag;
+  const uint32_t bar = sm100::smem_u32(&barrier);
+  if (threadIdx.x == 0) {
+    sm100::mbar_init(bar, 1);
+    abort_flag = 0;
+    sm100::mbar_init_fence();
+  }
+  __syncthreads();
+  sm100::WaitCtx wc{&abort_flag, dev_status, limit_ns};
+  const bool first = sm100::mbar_wait(bar, 0, wc);    // runs out
+  const bool second = sm100::mbar_wait(bar, 0, wc);   // returns at once: the CTA has given up
+  if (threadIdx.x == 0) *waits_returned = (first ? 1 : 0) + (second ? 2 : 0) + (abort_flag ? 4 : 0);
+}
+
+rf_status rf_launch_selftest_timeout(int32_t* dev_status, uint64_t limit_ns, int32_t* waits_returned, cudaStream_t st) {
+  rf_selftest_timeout_kernel<<<1, 32, 0, st>>>(dev_status, limit_ns, waits_returned);
+  return cudaGetLastError() == cudaSuccess ? RF_OK : RF_ERR_CUDA;
+}
+
 rf_status rf_launch_attention(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st) {
   switch (a.g.D) {
     case 64: return launch<64>(a, maps, st);

@@ -69,3 +69,4 @@ struct RfAttnArgs {
 // Tensor maps: [0..2] Q/K/V in original order, [3..5] the workspace copies with N rows per head
 // (position-major Q/K/V of Temporal heads), [6..7] workspace K/V with LkvTex rows per head (Textural).
 rf_status rf_launch_attention(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st);
+rf_status rf_launch_selftest_timeout(int32_t* dev_status, uint64_t limit_ns, int32_t* waits_returned, cudaStream_t st);

@@ -45,9 +45,10 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 struct WaitCtx {
   volatile int* abort_flag;  // shared memory, CTA-wide
   int32_t* dev_status;       // global, may be null
+  uint64_t limit_ns = 2000000000ull;   // wall-clock bound of one wait
 };
 
-// Bounded wait: two seconds of wall clock (and an iteration cap) at most.  Returns false if the wait
+// Bounded wait: w.limit_ns of wall clock (two seconds by default) and an iteration cap at most.  Returns false if the wait
 // was abandoned; from then on every wait of the CTA returns at once.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
   if (mbar_try(bar, parity)) return true;
@@ -55,7 +56,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
   for (uint32_t it = 0; it < (1u << 26); ++it) {
     if (mbar_try(bar, parity)) return true;
     if (*w.abort_flag) return false;
-    if (global_timer_ns() - t0 > 2000000000ull) break;
+    if (global_timer_ns() - t0 > w.limit_ns) break;
   }
   *w.abort_flag = 1;
   rf_report(w.dev_status, RF_ERR_TIMEOUT);

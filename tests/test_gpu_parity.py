@@ -259,3 +259,21 @@ def test_scores_with_large_dynamic_range_do_not_overflow():
     for h, cls in enumerate([D_, S_]):
         Or, lr = orc.masked_attention(qb, kb, v, cls, gu.geom(wl), gu.pparams(wl))
         gu.check_attention(O[0, h], lse[0, h], Or, lr, f"range class {cls}", strict=False)
+
+
+def test_bounded_wait_runs_out_cleanly_and_the_context_stays_usable():
+    """Failure detection without a fault: a wait on a barrier nobody arrives at gives up after its limit,
+    reports RF_ERR_TIMEOUT, later waits of the CTA return at once, the kernel exits, and the next real
+    call on the same context works."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ret = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    api.rf_selftest_wait_timeout(status, 20, ret)
+    t1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 5            # RF_ERR_TIMEOUT
+    assert int(ret.item()) == 4               # neither wait succeeded; abort flag set
+    assert 15.0 <= t0.elapsed_time(t1) <= 500.0
+    test_dense_tiny()                         # the context is intact

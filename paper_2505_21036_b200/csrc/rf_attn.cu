@@ -36,8 +36,12 @@ struct Cfg {
   static constexpr int COL1 = 64;
   static constexpr uint32_t BLK = 128 * 128;          // bytes of one 128-row x 64-col bf16 block
   static constexpr uint32_t TILE = KB * BLK;          // bytes of one 128-row tile
-  static constexpr int NK = D == 64 ? 4 : 2;          // K ring depth
-  static constexpr int NV = D == 64 ? 4 : 3;          // V ring depth
+  // D = 64 leaves room in shared memory for P (2 x 32 KB): the S accumulator is then free again as soon
+  // as the softmax warps have read it and the next tile's scores are computed during the softmax of the
+  // current one.  At D = 96 / 128 P lives in TMEM, on top of the S columns it was computed from.
+  static constexpr bool P_SMEM = D == 64;
+  static constexpr int NK = D == 64 ? 3 : 2;          // K ring depth
+  static constexpr int NV = D == 64 ? 3 : 2;          // V ring depth
   // byte offset, inside a tile, of the 16 columns of k-step ks of the Q K^T contraction
   static __host__ __device__ constexpr uint32_t koff(int ks) {
     return ks < 4 ? (uint32_t)ks * 32u : BLK + (uint32_t)(ks - 4) * 32u;
@@ -45,10 +49,12 @@ struct Cfg {
   static constexpr uint32_t Q = 0;
   static constexpr uint32_t K0 = Q + 2 * TILE;
   static constexpr uint32_t V0 = K0 + NK * TILE;
-  static constexpr uint32_t BAR = V0 + NV * TILE;
+  // P_SMEM only: [stream][two 64-key blocks of 128 rows x 128 B]
+  static constexpr uint32_t P0 = V0 + NV * TILE;
+  static constexpr uint32_t BAR = P0 + (P_SMEM ? 4 * BLK : 0);
   // barrier slots (8 bytes each)
   static constexpr int B_Q = 0, B_KF = 1, B_KE = B_KF + NK, B_VF = B_KE + NK, B_VE = B_VF + NV, B_SF = B_VE + NV,
-                       B_PF = B_SF + 2, B_OF = B_PF + 2, B_COUNT = B_OF + 2;
+                       B_PF = B_SF + 2, B_OF = B_PF + 2, B_SE = B_OF + 2 /* S read, P_SMEM only */, B_COUNT = B_SE + 2;
   static constexpr uint32_t MISC = BAR + 8 * ((B_COUNT + 7) / 8 * 8);
   static constexpr uint32_t TOTAL = MISC + 64;
   static constexpr uint32_t ALLOC = TOTAL + 1024;     // slack for manual 1024-byte alignment
@@ -221,6 +227,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       mbar_init(bar(C::B_SF + j), 1);
       mbar_init(bar(C::B_PF + j), 4);   // one arrival per softmax warp
       mbar_init(bar(C::B_OF + j), 1);
+      mbar_init(bar(C::B_SE + j), 4);
     }
     *abort_flag = 0;
     mbar_init_fence();
@@ -283,12 +290,17 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
                  IDESC_S, k > 0);
         tc_commit(bar(C::B_SF + j));
       };
+      const uint32_t p_lo = ((base + C::P0) >> 4) | LO_KMAJOR;
       auto issue_pv = [&](int j, int vs, bool first) {
         const uint32_t b0 = v_lo + vs * (C::TILE >> 4);
         const uint32_t t_p = tmem_base + (j ? C::S_COL1 : C::S_COL0), t_o = tmem_base + (j ? C::O_COL1 : C::O_COL0);
 #pragma unroll
         for (int k = 0; k < BN / 16; ++k) {
-          mma_ts(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
+          if constexpr (C::P_SMEM)
+            mma_ss(t_o, desc(p_lo + j * ((2 * C::BLK) >> 4) + (((k >> 2) * C::BLK + (k & 3) * 32) >> 4)),
+                   desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
+          else
+            mma_ts(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
         }
         tc_commit(bar(C::B_OF + j));
       };
@@ -297,12 +309,13 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       int cur_tile, cur_uses, nxt_tile = 0, nxt_uses = 0;
       bool has_cur = mg.next(L, cur_tile, cur_uses);
       int pv_cnt[2] = {0, 0};
+      int s_cnt[2] = {0, 0};   // P_SMEM: S tiles issued per stream
       mbar_wait(bar(C::B_Q), 0, wc);
       if (has_cur) {
         mbar_wait(bar(C::B_KF + 0), 0, wc);
         tc_fence_after();
-        if (cur_uses & 1) issue_s(0, 0);
-        if (cur_uses & 2) issue_s(1, 0);
+        if (cur_uses & 1) { issue_s(0, 0); ++s_cnt[0]; }
+        if (cur_uses & 2) { issue_s(1, 0); ++s_cnt[1]; }
         tc_commit(bar(C::B_KE + 0));
       }
       for (int u = 0; has_cur; ++u) {
@@ -312,15 +325,37 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         // keeps them out of the gap between a stream's P arriving and its MMAs being issued
         mbar_wait(bar(C::B_VF + vs), (u / C::NV) & 1, wc);
         if (has_nxt) mbar_wait(bar(C::B_KF + ksn), ((u + 1) / C::NK) & 1, wc);
+        if constexpr (C::P_SMEM) {
+          // the next tile's scores first: S is free as soon as the softmax warps have read the current one
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          if (cur_uses & (1 << j)) {
-            mbar_wait(bar(C::B_PF + j), pv_cnt[j] & 1, wc);
-            tc_fence_after();
-            issue_pv(j, vs, pv_cnt[j] == 0);
-            ++pv_cnt[j];
+          for (int j = 0; j < 2; ++j) {
+            if (has_nxt && (nxt_uses & (1 << j))) {
+              mbar_wait(bar(C::B_SE + j), (s_cnt[j] - 1) & 1, wc);
+              tc_fence_after();
+              issue_s(j, ksn);
+              ++s_cnt[j];
+            }
           }
-          if (has_nxt && (nxt_uses & (1 << j))) issue_s(j, ksn);
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (cur_uses & (1 << j)) {
+              mbar_wait(bar(C::B_PF + j), pv_cnt[j] & 1, wc);
+              tc_fence_after();
+              issue_pv(j, vs, pv_cnt[j] == 0);
+              ++pv_cnt[j];
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (cur_uses & (1 << j)) {
+              mbar_wait(bar(C::B_PF + j), pv_cnt[j] & 1, wc);
+              tc_fence_after();
+              issue_pv(j, vs, pv_cnt[j] == 0);
+              ++pv_cnt[j];
+            }
+            if (has_nxt && (nxt_uses & (1 << j))) issue_s(j, ksn);
+          }
         }
         tc_commit(bar(C::B_VE + vs));
         if (has_nxt) tc_commit(bar(C::B_KE + ksn));
@@ -351,6 +386,92 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       const int u0 = (int)(entry & ~RF_PARTIAL_BIT) * BN;
       mbar_wait(bar(C::B_SF + j), it & 1, wc);
       tc_fence_after();
+      if constexpr (C::P_SMEM) {
+        // S into registers, accumulator handed back at once; exact row maximum first (the scores are
+        // gone from TMEM, so there is no second pass), then one pass of exponentials into shared memory.
+        uint32_t s[128];
+        {
+          uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+          uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+          uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+          uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+          tmem_ld32(t_s, s0);
+          tmem_ld32(t_s + 32, s1);
+          tmem_ld32(t_s + 64, s2);
+          tmem_ld32(t_s + 96, s3);
+          tc_wait_ld();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C::B_SE + j));
+        if (partial) {
+          uint32_t w[4];
+          rmask.tile_bits(u0, w);
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (!((w[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf
+        }
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 128; c += 4) {
+          mx0 = fmaxf(mx0, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
+          mx1 = fmaxf(mx1, fmaxf(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])));
+        }
+        const float m_tile = fmaxf(mx0, mx1) * sc;
+        const bool raise = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
+        const bool any_raise = __any_sync(0xffffffffu, raise);
+        float alpha = 1.f;
+        if (raise) {
+          alpha = ex2(m_run - m_tile);   // 0 when m_run = -inf
+          m_run = m_tile;
+          l_run *= alpha;
+        }
+        if (it > 0) {
+          // P V of the previous tile reads the shared-memory P this tile is about to overwrite, and O may
+          // only be rescaled once everything issued into it has landed.  Waiting here also keeps this stream
+          // at most one tile ahead of the MMA warp, which tracks the P barrier by phase parity.
+          mbar_wait(bar(C::B_OF + j), (it - 1) & 1, wc);
+          if (any_raise) {
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t v[32];
+              tmem_ld32(t_o + c * 32, v);
+              tc_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+              tmem_st32(t_o + c * 32, v);
+            }
+            tc_wait_st();
+            tc_fence_before();
+          }
+        }
+        const float m_use = m_run == -INFINITY ? 0.f : m_run;
+        const float2 sc2 = make_float2(sc, sc), mneg = make_float2(-m_use, -m_use);
+        float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+        const uint32_t p_row = base + C::P0 + j * 2 * C::BLK + row_in_tile * 128;
+#pragma unroll
+        for (int c = 0; c < 128; c += 8) {
+          float2 e[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            e[i] = __ffma2_rn(make_float2(__uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1])), sc2, mneg);
+            e[i].x = ex2(e[i].x);
+            e[i].y = ex2(e[i].y);
+            if (i & 1) lb = __fadd2_rn(lb, e[i]); else la = __fadd2_rn(la, e[i]);
+          }
+          // 8 keys = one 16-byte chunk of the row; 128-byte swizzle: chunk index XOR (row mod 8)
+          const uint32_t chunk = (uint32_t)((c >> 3) & 7) ^ (uint32_t)(row_in_tile & 7);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_row + (c >> 6) * C::BLK + (chunk << 4)),
+                       "r"(pack_bf16(e[0].x, e[0].y)), "r"(pack_bf16(e[1].x, e[1].y)), "r"(pack_bf16(e[2].x, e[2].y)),
+                       "r"(pack_bf16(e[3].x, e[3].y)) : "memory");
+        }
+        l_run += (la.x + la.y) + (lb.x + lb.y);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C::B_PF + j));
+        continue;
+      }
       // Exponentials are taken against the running maximum of the previous tiles while the tile's own
       // maximum is computed alongside; only if some row's maximum grew by more than the threshold
       // (rare after the first tile) is the running maximum raised, O rescaled and the pass repeated

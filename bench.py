@@ -298,6 +298,23 @@ def run_cuda(args, wl):
                          "peak_kind": f"bf16 sustained, of {pk['source']}", "frac_of_burst": achieved / pk["bf16_burst"],
                          "algorithmic_flops_per_launch": tile_flops},
         }
+        # the small kernels against the HBM roofline (algorithmic bytes / measured time)
+        nS, nT, nX = (int((cls == c).sum()) for c in (0, 1, 2))
+        head_bytes = wl.N * wl.D * 2
+        n_glb = -(-wl.Nv // wl.sample_stride)
+        arm_bytes = wl.B * wl.H * 2 * (n_glb + (wl.S if wl.sample_mode == 0 else 0)) * wl.D * 2
+        mask_bytes = 4 * listed + 4 * wl.B * wl.H * sched.nQ
+        kept = sum(-(-(wl.frame_h - r) // wl.textural_stride) * -(-(wl.frame_w - r) // wl.textural_stride)
+                   for r in range(min(wl.textural_stride, wl.frame_h, wl.frame_w)))
+        tex_rows = wl.T * kept + wl.L_text
+        reorder_bytes = nT * 3 * 2 * head_bytes + nX * 2 * (head_bytes + tex_rows * wl.D * 2)
+        line["aux_kernels"] = {
+            name: {"ms": ms, "algorithmic_bytes": int(nbytes), "achieved_gbs": nbytes / (ms * 1e-3) / 1e9,
+                   "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "bound": bound}
+            for name, ms, nbytes, bound in (
+                ("rf_arm_classify", arm_ms, arm_bytes, "exponentials / tensor (n/2 flop per byte), not HBM"),
+                ("rf_build_block_mask", mask_ms, mask_bytes, "latency (closed-form integer work, 4 B per listed tile)"),
+                ("rf_reorder_tokens", reorder_ms, reorder_bytes, "hbm"))}
         if not args.no_cpu:
             dt, fl, nrows = oracle_sample(wl, args.ref_rows)
             line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads_used(), "kind": "oracle",

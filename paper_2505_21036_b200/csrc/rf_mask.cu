@@ -60,18 +60,19 @@ __device__ int tile_flag(const RfGeom& g, int cls, int a, int b) {
   return (all && full_width) ? 2 : 1;
 }
 
-// One CTA per (query tile, head): flags for all key tiles, then an ordered compaction.
+// One warp per (query tile, head): flags for 32 key tiles at a time, ordered compaction by ballot.
+// No block-level synchronisation; eight rows per CTA.
 __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int32_t* __restrict__ head_class,
                                                               const int32_t* __restrict__ head_window,
                                                               int32_t* __restrict__ count, int32_t* __restrict__ kv_tile,
                                                               uint32_t* __restrict__ bitmap, int32_t* __restrict__ kv_len,
                                                               int32_t* dev_status) {
-  __shared__ int warp_tot[8];
-  __shared__ int base;
-  const int a = blockIdx.x, bh = blockIdx.y;
+  const int lane = threadIdx.x & 31;
+  const int a = blockIdx.x * 8 + (threadIdx.x >> 5), bh = blockIdx.y;
+  if (a >= g.nQ) return;   // whole warp
   int cls = head_class[bh];
   if (cls < 0 || cls > 3) {
-    if (threadIdx.x == 0) rf_report(dev_status, RF_ERR_INVALID_ARG);
+    if (lane == 0) rf_report(dev_status, RF_ERR_INVALID_ARG);
     cls = RF_DENSE;
   }
   if (head_window != nullptr) {   // dynamic bandwidth: this head's own window
@@ -81,32 +82,20 @@ __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int
   }
   const int Lkv = rf_kv_len(g, cls);
   const int nK = rf_cdiv(Lkv, g.BN);
-  if (a == 0 && threadIdx.x == 0) kv_len[bh] = Lkv;
+  if (a == 0 && lane == 0) kv_len[bh] = Lkv;
   int32_t* row = kv_tile + ((size_t)bh * g.nQ + a) * g.nKmax;
   const int words = rf_cdiv(g.nKmax, 32);
   uint32_t* brow = bitmap ? bitmap + ((size_t)bh * g.nQ + a) * words : nullptr;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) base = 0;
-  __syncthreads();
-  for (int b0 = 0; b0 < g.nKmax; b0 += 256) {
-    const int b = b0 + threadIdx.x;
+  int base = 0;
+  for (int b0 = 0; b0 < words * 32; b0 += 32) {
+    const int b = b0 + lane;
     const int f = (b < nK) ? tile_flag(g, cls, a, b) : 0;
     const unsigned m = __ballot_sync(0xffffffffu, f != 0);
-    if (lane == 0) warp_tot[warp] = __popc(m);
-    if (brow && lane == 0 && (b >> 5) < words) brow[b >> 5] = m;
-    __syncthreads();
-    int off = base;
-    for (int w = 0; w < warp; ++w) off += warp_tot[w];
-    if (f != 0) row[off + __popc(m & ((1u << lane) - 1))] = (int32_t)((uint32_t)b | (f == 1 ? RF_PARTIAL_BIT : 0u));
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int t = 0;
-      for (int w = 0; w < 8; ++w) t += warp_tot[w];
-      base += t;
-    }
-    __syncthreads();
+    if (brow && lane == 0) brow[b0 >> 5] = m;
+    if (f != 0) row[base + __popc(m & ((1u << lane) - 1))] = (int32_t)((uint32_t)b | (f == 1 ? RF_PARTIAL_BIT : 0u));
+    base += __popc(m);
   }
-  if (threadIdx.x == 0) count[(size_t)bh * g.nQ + a] = base;
+  if (lane == 0) count[(size_t)bh * g.nQ + a] = base;
 }
 
 // Reordered copies for heads whose coordinate space is not the original one.
@@ -164,7 +153,7 @@ __global__ void __launch_bounds__(256) rf_gather_kernel(RfGeom g, const int32_t*
 
 cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, const int32_t* head_window, int32_t* count,
                                   int32_t* kv_tile, uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st) {
-  dim3 grid(g.nQ, g.B * g.H);
+  dim3 grid(rf_cdiv(g.nQ, 8), g.B * g.H);
   rf_build_tiles_kernel<<<grid, 256, 0, st>>>(g, head_class, head_window, count, kv_tile, bitmap, kv_len, dev_status);
   return cudaGetLastError();
 }

@@ -277,3 +277,28 @@ def test_bounded_wait_runs_out_cleanly_and_the_context_stays_usable():
     assert int(ret.item()) == 4               # neither wait succeeded; abort flag set
     assert 15.0 <= t0.elapsed_time(t1) <= 500.0
     test_dense_tiny()                         # the context is intact
+
+
+@pytest.mark.parametrize("D", [64, 96, 128])
+def test_attention_is_bit_reproducible(D):
+    """Same inputs, same schedule: every output bit must repeat (no races between the warp roles, no
+    order-dependent accumulation), for the sparse and the dense entry points, across many launches."""
+    wl = mid_workload(D=D)
+    run = gu.Run(wl)
+    run.force_classes([S_, T_, X_, D_])
+    run.build()
+    outs = []
+    for _ in range(4):
+        o = torch.empty((wl.B, wl.H, wl.N, wl.D), dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty((wl.B, wl.H, wl.N), dtype=torch.float32, device="cuda")
+        api.rf_sparse_attn_fwd(run.shape, run.params, run.q, run.k, run.v, run.head_class, run.sched, o, lse, run.ws,
+                               run.status)
+        od = torch.empty_like(o)
+        api.rf_dense_attn_fwd(run.shape, run.q, run.k, run.v, od, None, run.status)
+        outs.append((o, lse, od))
+    torch.cuda.synchronize()
+    assert int(run.status.item()) == 0
+    for o, lse, od in outs[1:]:
+        assert torch.equal(o.view(torch.int16), outs[0][0].view(torch.int16))
+        assert torch.equal(lse.view(torch.int32), outs[0][1].view(torch.int32))
+        assert torch.equal(od.view(torch.int16), outs[0][2].view(torch.int16))

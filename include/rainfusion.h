@@ -140,6 +140,18 @@ rf_status rf_reorder_tokens(const rf_shape *shape, const rf_params *params, cons
                             const void *v, const int32_t *head_class, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The attention kernel of rf_sparse_attn_fwd on its own (Eq. 1-2 under the masks of Eq. 3 and Eq. 5): the same
+ * arguments as rf_sparse_attn_fwd_plus (head_window may be NULL), but no reordering pass is launched.  ws must
+ * hold what rf_reorder_tokens wrote for the same q, k, v and head_class, earlier on the same stream.
+ * rf_reorder_tokens followed by this call is rf_sparse_attn_fwd, bit for bit; the split lets a caller reuse
+ * one reordering for several calls and lets each of the two kernels be timed by itself.
+ */
+rf_status rf_sparse_attn_reordered(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
+                                   const void *v, const int32_t *head_class, const int32_t *head_window,
+                                   const rf_schedule *sched, void *o, float *lse, void *ws, size_t ws_bytes,
+                                   int32_t *dev_status, void *cuda_stream);
+
+/*
  * Self-test of the device-side failure handling (no counterpart in the paper).  Every wait inside the kernels
  * (on TMA data, on the tensor cores, on another warp role) is bounded; when one runs out the CTA stops waiting,
  * reports RF_ERR_TIMEOUT through dev_status and still terminates normally.  This entry point launches one warp

@@ -19,7 +19,8 @@ _lib = None
 
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
            "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
-           "rf_arm_classify_noalloc", "rf_selftest_wait_timeout", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus"]
+           "rf_arm_classify_noalloc", "rf_selftest_wait_timeout", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus",
+           "rf_sparse_attn_reordered"]
 
 
 class rf_shape(C.Structure):
@@ -74,6 +75,8 @@ def load():
     lib.rf_build_block_mask_plus.argtypes = [P(rf_shape), P(rf_params), V, V, P(rf_schedule), V, V]
     lib.rf_sparse_attn_fwd_plus.restype = I
     lib.rf_sparse_attn_fwd_plus.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
+    lib.rf_sparse_attn_reordered.restype = I
+    lib.rf_sparse_attn_reordered.argtypes = lib.rf_sparse_attn_fwd_plus.argtypes
     lib.rf_selftest_wait_timeout.restype = I
     lib.rf_selftest_wait_timeout.argtypes = [V, C.c_int32, V, V]
     lib.rf_reorder_tokens.restype = I
@@ -196,6 +199,13 @@ def rf_sparse_attn_fwd_plus(shape, params, q, k, v, head_class, head_window, sch
                                           head_class.data_ptr(), _ptr(head_window), C.byref(sched.c), o.data_ptr(),
                                           _ptr(lse), ws.data_ptr(), ws.numel(), _ptr(dev_status), _stream()),
            "rf_sparse_attn_fwd_plus")
+
+
+def rf_sparse_attn_reordered(shape, params, q, k, v, head_class, head_window, sched: Schedule, o, lse, ws, dev_status=None):
+    _check(load().rf_sparse_attn_reordered(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                           head_class.data_ptr(), _ptr(head_window), C.byref(sched.c), o.data_ptr(),
+                                           _ptr(lse), ws.data_ptr(), ws.numel(), _ptr(dev_status), _stream()),
+           "rf_sparse_attn_reordered")
 
 
 def rf_selftest_wait_timeout(dev_status, limit_ms, waits_returned):

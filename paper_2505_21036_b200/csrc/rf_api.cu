@@ -115,6 +115,62 @@ rf_status rf_checked_geom(const rf_shape* shape, const rf_params* params, RfGeom
   return RF_OK;
 }
 
+namespace {
+// Shared by rf_sparse_attn_fwd(_plus) and rf_sparse_attn_reordered: the second skips the gather pass and
+// reads the reordered copies a preceding rf_reorder_tokens call left in the workspace.
+rf_status sparse_attn_impl(const rf_shape* shape, const rf_params* params, const void* q, const void* k, const void* v,
+                           const int32_t* head_class, const int32_t* head_window, const rf_schedule* sched, void* o,
+                           float* lse, void* ws, size_t ws_bytes, int32_t* dev_status, void* cuda_stream, bool gather) {
+  rf_status st = check_attn_shape(shape);
+  if (st != RF_OK) return st;
+  st = check_params(params);
+  if (st != RF_OK) return st;
+  if (params->block_m != 128 || params->block_n != 128) return RF_ERR_UNSUPPORTED;
+  if (q == nullptr || k == nullptr || v == nullptr || o == nullptr || head_class == nullptr || sched == nullptr ||
+      sched->count == nullptr || sched->kv_tile == nullptr || ws == nullptr)
+    return RF_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
+      (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0)
+    return RF_ERR_INVALID_ARG;
+  if (ws_bytes < rf_workspace_bytes(shape, params)) return RF_ERR_WORKSPACE_TOO_SMALL;
+  const RfGeom g = make_geom(shape, params);
+  if (sched->nQ != g.nQ || sched->nKmax != g.nKmax) return RF_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  __nv_bfloat16* wq = reinterpret_cast<__nv_bfloat16*>(w);
+  __nv_bfloat16* wk = reinterpret_cast<__nv_bfloat16*>(w + tensor_bytes(g));
+  __nv_bfloat16* wv = reinterpret_cast<__nv_bfloat16*>(w + 2 * tensor_bytes(g));
+
+  CUtensorMap maps[8];
+  const int heads = g.B * g.H;
+  bool ok = encode_map(&maps[0], q, g.D, g.N, g.N, heads) && encode_map(&maps[1], k, g.D, g.N, g.N, heads) &&
+            encode_map(&maps[2], v, g.D, g.N, g.N, heads) && encode_map(&maps[3], wq, g.D, g.N, g.N, heads) &&
+            encode_map(&maps[4], wk, g.D, g.N, g.N, heads) && encode_map(&maps[5], wv, g.D, g.N, g.N, heads) &&
+            encode_map(&maps[6], wk, g.D, g.LkvTex, g.N, heads) && encode_map(&maps[7], wv, g.D, g.LkvTex, g.N, heads);
+  if (!ok) return RF_ERR_CUDA;
+
+  if (gather) {
+    cudaError_t e = rf_launch_gather(g, head_class, static_cast<const __nv_bfloat16*>(q),
+                                     static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), wq, wk, wv,
+                                     stream);
+    if (e != cudaSuccess) return RF_ERR_CUDA;
+  }
+
+  RfAttnArgs a;
+  a.g = g;
+  a.head_class = head_class;
+  a.head_window = head_window;
+  a.count = sched->count;
+  a.kv_tile = sched->kv_tile;
+  a.o = static_cast<__nv_bfloat16*>(o);
+  a.lse = lse;
+  a.dev_status = dev_status;
+  a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.D);
+  return rf_launch_attention(a, maps, stream);
+}
+}  // namespace
+
 extern "C" {
 
 const char* rf_status_string(rf_status s) {
@@ -224,50 +280,16 @@ rf_status rf_sparse_attn_fwd_plus(const rf_shape* shape, const rf_params* params
                                   const void* v, const int32_t* head_class, const int32_t* head_window,
                                   const rf_schedule* sched, void* o, float* lse, void* ws, size_t ws_bytes,
                                   int32_t* dev_status, void* cuda_stream) {
-  rf_status st = check_attn_shape(shape);
-  if (st != RF_OK) return st;
-  st = check_params(params);
-  if (st != RF_OK) return st;
-  if (params->block_m != 128 || params->block_n != 128) return RF_ERR_UNSUPPORTED;
-  if (q == nullptr || k == nullptr || v == nullptr || o == nullptr || head_class == nullptr || sched == nullptr ||
-      sched->count == nullptr || sched->kv_tile == nullptr || ws == nullptr)
-    return RF_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
-      (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0)
-    return RF_ERR_INVALID_ARG;
-  if (ws_bytes < rf_workspace_bytes(shape, params)) return RF_ERR_WORKSPACE_TOO_SMALL;
-  const RfGeom g = make_geom(shape, params);
-  if (sched->nQ != g.nQ || sched->nKmax != g.nKmax) return RF_ERR_INVALID_ARG;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  return sparse_attn_impl(shape, params, q, k, v, head_class, head_window, sched, o, lse, ws, ws_bytes, dev_status,
+                          cuda_stream, true);
+}
 
-  uint8_t* w = static_cast<uint8_t*>(ws);
-  __nv_bfloat16* wq = reinterpret_cast<__nv_bfloat16*>(w);
-  __nv_bfloat16* wk = reinterpret_cast<__nv_bfloat16*>(w + tensor_bytes(g));
-  __nv_bfloat16* wv = reinterpret_cast<__nv_bfloat16*>(w + 2 * tensor_bytes(g));
-
-  CUtensorMap maps[8];
-  const int heads = g.B * g.H;
-  bool ok = encode_map(&maps[0], q, g.D, g.N, g.N, heads) && encode_map(&maps[1], k, g.D, g.N, g.N, heads) &&
-            encode_map(&maps[2], v, g.D, g.N, g.N, heads) && encode_map(&maps[3], wq, g.D, g.N, g.N, heads) &&
-            encode_map(&maps[4], wk, g.D, g.N, g.N, heads) && encode_map(&maps[5], wv, g.D, g.N, g.N, heads) &&
-            encode_map(&maps[6], wk, g.D, g.LkvTex, g.N, heads) && encode_map(&maps[7], wv, g.D, g.LkvTex, g.N, heads);
-  if (!ok) return RF_ERR_CUDA;
-
-  cudaError_t e = rf_launch_gather(g, head_class, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
-                                   static_cast<const __nv_bfloat16*>(v), wq, wk, wv, stream);
-  if (e != cudaSuccess) return RF_ERR_CUDA;
-
-  RfAttnArgs a;
-  a.g = g;
-  a.head_class = head_class;
-  a.head_window = head_window;
-  a.count = sched->count;
-  a.kv_tile = sched->kv_tile;
-  a.o = static_cast<__nv_bfloat16*>(o);
-  a.lse = lse;
-  a.dev_status = dev_status;
-  a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.D);
-  return rf_launch_attention(a, maps, stream);
+rf_status rf_sparse_attn_reordered(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
+                                   const void* v, const int32_t* head_class, const int32_t* head_window,
+                                   const rf_schedule* sched, void* o, float* lse, void* ws, size_t ws_bytes,
+                                   int32_t* dev_status, void* cuda_stream) {
+  return sparse_attn_impl(shape, params, q, k, v, head_class, head_window, sched, o, lse, ws, ws_bytes, dev_status,
+                          cuda_stream, false);
 }
 
 rf_status rf_selftest_wait_timeout(int32_t* dev_status, int32_t limit_ms, int32_t* waits_returned, void* cuda_stream) {

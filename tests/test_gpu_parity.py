@@ -302,3 +302,29 @@ def test_attention_is_bit_reproducible(D):
         assert torch.equal(o.view(torch.int16), outs[0][0].view(torch.int16))
         assert torch.equal(lse.view(torch.int32), outs[0][1].view(torch.int32))
         assert torch.equal(od.view(torch.int16), outs[0][2].view(torch.int16))
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_reorder_then_attention_equals_the_fused_call(D):
+    """rf_reorder_tokens + rf_sparse_attn_reordered launch the same two kernels as rf_sparse_attn_fwd."""
+    wl = mid_workload(D=D)
+    run = gu.Run(wl)
+    run.force_classes([S_, T_, X_, D_])
+    run.build()
+
+    def outputs():
+        o = torch.full((wl.B, wl.H, wl.N, wl.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((wl.B, wl.H, wl.N), float("nan"), dtype=torch.float32, device="cuda")
+        return o, lse
+    o1, l1 = outputs()
+    api.rf_sparse_attn_fwd(run.shape, run.params, run.q, run.k, run.v, run.head_class, run.sched, o1, l1, run.ws, run.status)
+    run.ws.zero_()
+    o2, l2 = outputs()
+    api.rf_reorder_tokens(run.shape, run.params, run.q, run.k, run.v, run.head_class, run.ws)
+    for _ in range(2):   # one reordering serves several attention calls
+        api.rf_sparse_attn_reordered(run.shape, run.params, run.q, run.k, run.v, run.head_class, None, run.sched, o2, l2,
+                                     run.ws, run.status)
+    torch.cuda.synchronize()
+    assert int(run.status.item()) == 0
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+    assert torch.equal(l1.view(torch.int32), l2.view(torch.int32))

@@ -11,8 +11,10 @@
 // Per listed tile and stream: S lands in TMEM, the softmax warps read their rows (tcgen05.ld), keep a
 // running maximum and sum in fp32, write P as packed bf16 back into the S columns (tcgen05.st) and the
 // MMA warp multiplies it with V straight from TMEM.  The running maximum is only raised when it grows
-// by more than 2^8 (P stays well inside bf16/fp32 range), in which case the softmax warp itself
-// rescales its rows of O in TMEM; the final O / l and the log-sum-exp are exact either way.
+// by more than 2^32, in which case the softmax warp itself rescales its rows of O in TMEM.  bf16 P and
+// the fp32 sums carry the same relative precision at every exponent, and 2^32 times the longest row
+// is far from overflow, so the final O / l and the log-sum-exp are exact either way; with a small
+// threshold, inputs whose logits rise along the row would pay a second softmax pass for many tiles.
 // PARTIAL tiles apply the exact element mask of the head's pattern; FULL tiles skip it.
 #include "rf_sm100.cuh"
 
@@ -23,7 +25,13 @@ using namespace sm100;
 constexpr int BM = 128, BN = 128;
 constexpr int kThreads = 384;               // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
 constexpr int kTmaWarp = 8, kMmaWarp = 9;
-constexpr float kRescaleThreshold = 8.0f;  // log2 units
+// Lazy rescaling of the running maximum.  A tile's weights are taken as 2^(score - running maximum) and accepted
+// while their row sum stays within kSumLimit; beyond it the row's maximum is raised.  bf16 P and the fp32 sums
+// carry the same relative precision at every exponent and 2^32 times the longest row is far from overflow, so
+// O / l and the log-sum-exp do not depend on how stale the running maximum is.
+constexpr float kSumLimit = 4294967296.0f;  // 2^32
+constexpr float kRaiseMargin = 8.0f;        // log2 units: on the slow path, rows this far above their maximum raise it
+constexpr float kLazyRaise = 32.0f;         // log2 units: where the exact tile maximum is at hand (D = 64)
 
 struct Maps { CUtensorMap m[8]; };
 
@@ -61,6 +69,13 @@ struct Cfg {
   // TMEM columns
   static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL0 = 256, O_COL1 = 384, TMEM_COLS = 512;
 };
+
+// The two bf16 values of a packed word, widened exactly.  The row sum is taken over these rounded weights, the
+// ones the tensor core multiplies with V: O / l is then an exact convex combination of V rows with slightly
+// perturbed weights, and the rounding of a dominant weight cancels instead of scaling the whole output row.
+__device__ __forceinline__ float2 unpack_bf16(uint32_t w) {
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -130,6 +145,23 @@ __device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r
     }
   }
   return m;
+}
+
+// Exact maximum of this thread's row of the S tile at t_s (slow path of the softmax; warp-collective loads).
+__device__ __noinline__ float tile_row_max(uint32_t t_s, bool partial, const RowMask& rmask, int u0) {
+  uint32_t w[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+  if (partial) rmask.tile_bits(u0, w);
+  float mx = -INFINITY;
+#pragma unroll 1
+  for (int q = 0; q < 4; ++q) {
+    uint32_t v[32];
+    tmem_ld32(t_s + q * 32, v);
+    tc_wait_ld();
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+      if ((w[q] >> c) & 1u) mx = fmaxf(mx, __uint_as_float(v[c]));
+  }
+  return mx;
 }
 
 // The two streams' ascending tile lists and their merge (the order K/V tiles are fetched in).
@@ -378,7 +410,8 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
     const RowMask rmask = make_row_mask(g, cls, min(r, g.N - 1));
     const float sc = a.scale_log2;
     float m_run = -INFINITY;   // running maximum, log2 domain (score * sc)
-    float l_run = 0.f;
+    float l_run = 0.f;         // sum of the weights as rounded to bf16, the ones P V multiplies: normalises O
+    float l_exact = 0.f;       // sum of the unrounded weights: the log-sum-exp
 
     for (int it = 0; it < n; ++it) {
       const uint32_t entry = L.entry(j, it);
@@ -387,8 +420,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       mbar_wait(bar(C::B_SF + j), it & 1, wc);
       tc_fence_after();
       if constexpr (C::P_SMEM) {
-        // S into registers, accumulator handed back at once; exact row maximum first (the scores are
-        // gone from TMEM, so there is no second pass), then one pass of exponentials into shared memory.
+        // S into registers and the accumulator handed back at once; the exponentials go to shared memory.
         uint32_t s[128];
         {
           uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
@@ -411,6 +443,8 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           for (int c = 0; c < 128; ++c)
             if (!((w[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;  // -inf
         }
+        // The scores are gone from TMEM, so the exact row maximum comes first and the exponentials are
+        // taken once; the running maximum is raised only when the tile exceeds it by kLazyRaise.
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 128; c += 4) {
@@ -418,13 +452,14 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           mx1 = fmaxf(mx1, fmaxf(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])));
         }
         const float m_tile = fmaxf(mx0, mx1) * sc;
-        const bool raise = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
+        const bool raise = m_tile > m_run + kLazyRaise || (m_run == -INFINITY && m_tile > -INFINITY);
         const bool any_raise = __any_sync(0xffffffffu, raise);
         float alpha = 1.f;
         if (raise) {
           alpha = ex2(m_run - m_tile);   // 0 when m_run = -inf
           m_run = m_tile;
           l_run *= alpha;
+          l_exact *= alpha;
         }
         if (it > 0) {
           // P V of the previous tile reads the shared-memory P this tile is about to overwrite, and O may
@@ -452,30 +487,34 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         const uint32_t p_row = base + C::P0 + j * 2 * C::BLK + row_in_tile * 128;
 #pragma unroll
         for (int c = 0; c < 128; c += 8) {
-          float2 e[4];
+          uint32_t pw[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            e[i] = __ffma2_rn(make_float2(__uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1])), sc2, mneg);
-            e[i].x = ex2(e[i].x);
-            e[i].y = ex2(e[i].y);
-            if (i & 1) lb = __fadd2_rn(lb, e[i]); else la = __fadd2_rn(la, e[i]);
+            float2 e = __ffma2_rn(make_float2(__uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1])), sc2, mneg);
+            e.x = ex2(e.x);
+            e.y = ex2(e.y);
+            pw[i] = pack_bf16(e.x, e.y);
+            la = __fadd2_rn(la, e);
+            lb = __fadd2_rn(lb, unpack_bf16(pw[i]));
           }
           // 8 keys = one 16-byte chunk of the row; 128-byte swizzle: chunk index XOR (row mod 8)
           const uint32_t chunk = (uint32_t)((c >> 3) & 7) ^ (uint32_t)(row_in_tile & 7);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_row + (c >> 6) * C::BLK + (chunk << 4)),
-                       "r"(pack_bf16(e[0].x, e[0].y)), "r"(pack_bf16(e[1].x, e[1].y)), "r"(pack_bf16(e[2].x, e[2].y)),
-                       "r"(pack_bf16(e[3].x, e[3].y)) : "memory");
+                       "r"(pw[0]), "r"(pw[1]), "r"(pw[2]), "r"(pw[3]) : "memory");
         }
-        l_run += (la.x + la.y) + (lb.x + lb.y);
+        l_exact += la.x + la.y;
+        l_run += lb.x + lb.y;
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(C::B_PF + j));
         continue;
       }
-      // Exponentials are taken against the running maximum of the previous tiles while the tile's own
-      // maximum is computed alongside; only if some row's maximum grew by more than the threshold
-      // (rare after the first tile) is the running maximum raised, O rescaled and the pass repeated
-      // (S is still in TMEM then: P has not been stored yet).
+      // Exponentials are taken against the running maximum of the previous tiles, without looking at the
+      // tile's own maximum: all weights are non-negative, so a row sum within kSumLimit proves that none
+      // of them left the safe range.  Only if some row's sum does not (its maximum grew by more than
+      // ~2^25; rare after a row's first tile) is the exact tile maximum taken from the scores, which are
+      // still in TMEM because P has not been stored yet, the running maximum raised, O rescaled and the
+      // pass repeated.
       uint32_t pk[64];
 #pragma unroll 1
       for (int pass = 0; pass < 2; ++pass) {
@@ -501,32 +540,29 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         const float m_use = m_run == -INFINITY ? 0.f : m_run;
         const float2 sc2 = make_float2(sc, sc), mneg = make_float2(-m_use, -m_use);
         float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
-        float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 128; c += 4) {
-          const float s0 = __uint_as_float(s[c]), s1 = __uint_as_float(s[c + 1]);
-          const float s2 = __uint_as_float(s[c + 2]), s3 = __uint_as_float(s[c + 3]);
-          mx0 = fmaxf(mx0, fmaxf(s0, s1));
-          mx1 = fmaxf(mx1, fmaxf(s2, s3));
-          float2 e0 = __ffma2_rn(make_float2(s0, s1), sc2, mneg);
-          float2 e1 = __ffma2_rn(make_float2(s2, s3), sc2, mneg);
+          float2 e0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, mneg);
+          float2 e1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, mneg);
           e0.x = ex2(e0.x); e0.y = ex2(e0.y);
           e1.x = ex2(e1.x); e1.y = ex2(e1.y);
-          la = __fadd2_rn(la, e0);
-          lb = __fadd2_rn(lb, e1);
           pk[c / 2] = pack_bf16(e0.x, e0.y);
           pk[c / 2 + 1] = pack_bf16(e1.x, e1.y);
+          la = __fadd2_rn(la, __fadd2_rn(e0, e1));
+          lb = __fadd2_rn(lb, __fadd2_rn(unpack_bf16(pk[c / 2]), unpack_bf16(pk[c / 2 + 1])));
         }
-        const float l_tile = (la.x + la.y) + (lb.x + lb.y);
-        if (pass == 1) { l_run += l_tile; break; }
-        const float m_tile = fmaxf(mx0, mx1) * sc;
-        const bool raise = m_tile > m_run + kRescaleThreshold || (m_run == -INFINITY && m_tile > -INFINITY);
-        if (!__any_sync(0xffffffffu, raise)) { l_run += l_tile; break; }
+        const float l_tile = lb.x + lb.y, l_tile_exact = la.x + la.y;
+        if (pass == 1) { l_run += l_tile; l_exact += l_tile_exact; break; }
+        const bool bad = !(l_tile <= kSumLimit) || m_run == -INFINITY;
+        if (!__any_sync(0xffffffffu, bad)) { l_run += l_tile; l_exact += l_tile_exact; break; }
+        const float m_tile = tile_row_max(t_s, partial, rmask, u0) * sc;
+        const bool raise = m_tile > m_run + kRaiseMargin || (m_run == -INFINITY && m_tile > -INFINITY);
         float alpha = 1.f;
         if (raise) {
           alpha = ex2(m_run - m_tile);   // 0 when m_run = -inf
           m_run = m_tile;
           l_run *= alpha;
+          l_exact *= alpha;
         }
         if (it > 0) {
           // O of the previous tiles must be complete before it is rescaled
@@ -580,7 +616,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           }
         }
       }
-      if (r < g.N && a.lse != nullptr) a.lse[(size_t)bh * g.N + tok] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+      if (r < g.N && a.lse != nullptr) a.lse[(size_t)bh * g.N + tok] = (m_run + log2f(l_exact)) * 0.6931471805599453f;
     }
   }
 

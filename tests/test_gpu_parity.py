@@ -328,3 +328,45 @@ def test_reorder_then_attention_equals_the_fused_call(D):
     assert int(run.status.item()) == 0
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
     assert torch.equal(l1.view(torch.int32), l2.view(torch.int32))
+
+
+@pytest.mark.parametrize("D", [64, 96, 128])
+def test_row_maximum_growing_in_late_tiles(D):
+    """The running maximum is only raised (and O rescaled) when a tile's maximum exceeds it by a wide margin.
+    Here it does, repeatedly and at different tiles for neighbouring rows: even rows meet keys whose logit
+    steps up by ~30 nats in tiles 2 and 4, odd rows in tiles 1, 3 and 5; every earlier contribution must
+    then be scaled down by e^-30 in O and in the row sum alike."""
+    wl = mid_workload(D=D, H=2)
+    q, k, v = synth.make_head(wl, 0, 0, kind="none")
+    qf, kf, vf = (synth.bf16_bits_to_f32(x).copy() for x in (q, k, v))
+    qf *= 0.25
+    kf *= 0.25
+    N = wl.N
+    step = 30.0 * np.sqrt(D) / 8.0            # logit = 8 * level * step / sqrt(D) = 30 * level nats
+    qf[:, 0] = 0.0
+    qf[:, 1] = 0.0
+    qf[0::2, 0] = 8.0
+    qf[1::2, 1] = 8.0
+    kf[:, 0] = 0.0
+    kf[:, 1] = 0.0
+    rng = np.random.default_rng(11)
+    for level, t in enumerate((2, 4), start=1):           # feature 0: even rows
+        idx = t * 128 + rng.choice(128, size=5, replace=False)
+        kf[idx[idx < N], 0] = level * step
+    for level, t in enumerate((1, 3, 5), start=1):        # feature 1: odd rows
+        idx = t * 128 + rng.choice(128, size=5, replace=False)
+        kf[idx[idx < N], 1] = level * step
+    bits = tuple(synth.f32_to_bf16_bits(x) for x in (qf, kf, vf))
+    stack = tuple(np.stack([x, x])[None] for x in bits)
+    run = gu.Run(wl, qkv=stack)
+    run.force_classes([D_, X_])
+    run.build()
+    g, pp = gu.geom(wl), gu.pparams(wl)
+    O, lse = run.sparse()
+    Od, lsed = run.dense()
+    ref_d = orc.masked_attention(*bits, D_, g, pp)
+    ref_x = orc.masked_attention(*bits, X_, g, pp)
+    assert ref_d[1].max() > 80.0                       # the staircase really is there
+    gu.check_attention(O[0, 0], lse[0, 0], *ref_d, "staircase sparse/dense-class", strict=False)
+    gu.check_attention(O[0, 1], lse[0, 1], *ref_x, "staircase textural", strict=False)
+    gu.check_attention(Od[0, 1], lsed[0, 1], *ref_d, "staircase dense entry", strict=False)

@@ -61,7 +61,12 @@ struct Cfg {
   static constexpr uint32_t P0 = V0 + NV * TILE;
   static constexpr uint32_t BAR = P0 + (P_SMEM ? 4 * BLK : 0);
   // barrier slots (8 bytes each)
-  static constexpr int B_Q = 0, B_KF = 1, B_KE = B_KF + NK, B_VF = B_KE + NK, B_VE = B_VF + NV, B_SF = B_VE + NV,
+  // V of tile u and K of tile u + 1 travel as a pair: they are wanted in the same iteration of the MMA warp and
+  // released by it together, so one full and one empty barrier per pair (B_F, B_E) serve both; K of the first
+  // tile has its own two (B_K0 landed, B_K0E consumed).
+  static_assert(NK == NV, "K and V rings advance together");
+  static constexpr int NP = NV;
+  static constexpr int B_Q = 0, B_K0 = 1, B_K0E = 2, B_F = 3, B_E = B_F + NP, B_SF = B_E + NP,
                        B_PF = B_SF + 2, B_OF = B_PF + 2, B_SE = B_OF + 2 /* S read, P_SMEM only */, B_COUNT = B_SE + 2;
   static constexpr uint32_t MISC = BAR + 8 * ((B_COUNT + 7) / 8 * 8);
   static constexpr uint32_t TOTAL = MISC + 64;
@@ -253,8 +258,9 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
 
   if (tid == 0) {
     mbar_init(bar(C::B_Q), 1);
-    for (int s = 0; s < C::NK; ++s) { mbar_init(bar(C::B_KF + s), 1); mbar_init(bar(C::B_KE + s), 1); }
-    for (int s = 0; s < C::NV; ++s) { mbar_init(bar(C::B_VF + s), 1); mbar_init(bar(C::B_VE + s), 1); }
+    mbar_init(bar(C::B_K0), 1);
+    mbar_init(bar(C::B_K0E), 1);
+    for (int s = 0; s < C::NP; ++s) { mbar_init(bar(C::B_F + s), 1); mbar_init(bar(C::B_E + s), 1); }
     for (int j = 0; j < 2; ++j) {
       mbar_init(bar(C::B_SF + j), 1);
       mbar_init(bar(C::B_PF + j), 4);   // one arrival per softmax warp
@@ -288,19 +294,32 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           tma_load_3d(base + C::Q + j * C::TILE + kb * C::BLK, map_q, kb * C::COL1, (qt0 + j) * BM, bh, bar(C::B_Q));
       Merge mg;
       mg.start(L);
-      int tile, uses;
-      for (int u = 0; mg.next(L, tile, uses); ++u) {
-        const int ks = u % C::NK, vs = u % C::NV;
-        if (u >= C::NK) mbar_wait(bar(C::B_KE + ks), ((u / C::NK) - 1) & 1, wc);
-        mbar_expect_tx(bar(C::B_KF + ks), C::TILE);
+      int tile, uses, ntile = 0;
+      bool has = mg.next(L, tile, uses);
+      if (has) {
+        mbar_expect_tx(bar(C::B_K0), C::TILE);
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_3d(base + C::K0 + ks * C::TILE + kb * C::BLK, map_k, kb * C::COL1, tile * BN, bh, bar(C::B_KF + ks));
-        if (u >= C::NV) mbar_wait(bar(C::B_VE + vs), ((u / C::NV) - 1) & 1, wc);
-        mbar_expect_tx(bar(C::B_VF + vs), C::TILE);
+          tma_load_3d(base + C::K0 + kb * C::BLK, map_k, kb * C::COL1, tile * BN, bh, bar(C::B_K0));
+      }
+      for (int u = 0; has; ++u) {
+        const bool has_nxt = mg.next(L, ntile, uses);
+        const int ps = u % C::NP, ksn = (u + 1) % C::NK;
+        // pair u reuses the V slot of pair u - NP and the K slot that pair filled; the first tile's K slot
+        // comes round at u = NK - 1
+        if (u >= C::NP) mbar_wait(bar(C::B_E + ps), ((u / C::NP) - 1) & 1, wc);
+        else if (has_nxt && ksn == 0) mbar_wait(bar(C::B_K0E), 0, wc);
+        mbar_expect_tx(bar(C::B_F + ps), has_nxt ? 2 * C::TILE : C::TILE);
 #pragma unroll
         for (int kb = 0; kb < KB; ++kb)
-          tma_load_3d(base + C::V0 + vs * C::TILE + kb * C::BLK, map_v, kb * C::COL1, tile * BN, bh, bar(C::B_VF + vs));
+          tma_load_3d(base + C::V0 + ps * C::TILE + kb * C::BLK, map_v, kb * C::COL1, tile * BN, bh, bar(C::B_F + ps));
+        if (has_nxt) {
+#pragma unroll
+          for (int kb = 0; kb < KB; ++kb)
+            tma_load_3d(base + C::K0 + ksn * C::TILE + kb * C::BLK, map_k, kb * C::COL1, ntile * BN, bh, bar(C::B_F + ps));
+        }
+        has = has_nxt;
+        tile = ntile;
       }
     }
   } else if (warp == kMmaWarp) {
@@ -344,19 +363,18 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       int s_cnt[2] = {0, 0};   // P_SMEM: S tiles issued per stream
       mbar_wait(bar(C::B_Q), 0, wc);
       if (has_cur) {
-        mbar_wait(bar(C::B_KF + 0), 0, wc);
+        mbar_wait(bar(C::B_K0), 0, wc);
         tc_fence_after();
         if (cur_uses & 1) { issue_s(0, 0); ++s_cnt[0]; }
         if (cur_uses & 2) { issue_s(1, 0); ++s_cnt[1]; }
-        tc_commit(bar(C::B_KE + 0));
+        tc_commit(bar(C::B_K0E));
       }
       for (int u = 0; has_cur; ++u) {
         const bool has_nxt = mg.next(L, nxt_tile, nxt_uses);
         const int vs = u % C::NV, ksn = (u + 1) % C::NK;
-        // the TMA barriers first: their data has normally landed long ago, and checking them here
-        // keeps them out of the gap between a stream's P arriving and its MMAs being issued
-        mbar_wait(bar(C::B_VF + vs), (u / C::NV) & 1, wc);
-        if (has_nxt) mbar_wait(bar(C::B_KF + ksn), ((u + 1) / C::NK) & 1, wc);
+        // the TMA barrier first (V of this tile and K of the next): the data has normally landed long ago, and
+        // checking here keeps it out of the gap between a stream's P arriving and its MMAs being issued
+        mbar_wait(bar(C::B_F + vs), (u / C::NP) & 1, wc);
         if constexpr (C::P_SMEM) {
           // the next tile's scores first: S is free as soon as the softmax warps have read the current one
 #pragma unroll
@@ -389,8 +407,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
             if (has_nxt && (nxt_uses & (1 << j))) issue_s(j, ksn);
           }
         }
-        tc_commit(bar(C::B_VE + vs));
-        if (has_nxt) tc_commit(bar(C::B_KE + ksn));
+        tc_commit(bar(C::B_E + vs));
         has_cur = has_nxt;
         cur_tile = nxt_tile;
         cur_uses = nxt_uses;

@@ -5,16 +5,15 @@
 // contractions.  Warp roles:
 //   warps 0-3  softmax of stream 0   (one thread per query row, TMEM lane = row)
 //   warps 4-7  softmax of stream 1
-//   warp  8    TMA producer: Q once, then K and V tiles into two shared-memory rings
+//   warp  8    TMA producer: Q once, then K and V tiles into two shared-memory rings (V of tile u and K of
+//              tile u + 1 as a pair under one full / one empty mbarrier)
 //   warp  9    MMA issuer: tcgen05.mma, accumulators in TMEM (S0, S1, O0, O1)
 //   (warps 10-11 only fill the third warpgroup, which hands its registers to the softmax warpgroups)
 // Per listed tile and stream: S lands in TMEM, the softmax warps read their rows (tcgen05.ld), keep a
-// running maximum and sum in fp32, write P as packed bf16 back into the S columns (tcgen05.st) and the
-// MMA warp multiplies it with V straight from TMEM.  The running maximum is only raised when it grows
-// by more than 2^32, in which case the softmax warp itself rescales its rows of O in TMEM.  bf16 P and
-// the fp32 sums carry the same relative precision at every exponent, and 2^32 times the longest row
-// is far from overflow, so the final O / l and the log-sum-exp are exact either way; with a small
-// threshold, inputs whose logits rise along the row would pay a second softmax pass for many tiles.
+// running maximum and sum in fp32, write P as packed bf16 back into TMEM (tcgen05.st: on top of the S
+// columns at D = 96 / 128, into spare columns at D = 64) and the MMA warp multiplies it with V straight
+// from TMEM.  The running maximum is raised lazily (see kSumLimit), in which case the softmax warp itself
+// rescales its rows of O in TMEM; the final O / l and the log-sum-exp do not depend on it.
 // PARTIAL tiles apply the exact element mask of the head's pattern; FULL tiles skip it.
 #include "rf_sm100.cuh"
 
@@ -44,10 +43,11 @@ struct Cfg {
   static constexpr int COL1 = 64;
   static constexpr uint32_t BLK = 128 * 128;          // bytes of one 128-row x 64-col bf16 block
   static constexpr uint32_t TILE = KB * BLK;          // bytes of one 128-row tile
-  // D = 64 leaves room in shared memory for P (2 x 32 KB): the S accumulator is then free again as soon
-  // as the softmax warps have read it and the next tile's scores are computed during the softmax of the
-  // current one.  At D = 96 / 128 P lives in TMEM, on top of the S columns it was computed from.
-  static constexpr bool P_SMEM = D == 64;
+  // D = 64 leaves 128 TMEM columns unused (O is only 64 wide), room for P of both streams in columns of its
+  // own: the S accumulator is then free again as soon as the softmax warps have read it, and the next tile's
+  // scores are computed during the softmax of the current one.  At D = 96 / 128 TMEM is full and P lives on
+  // top of the S columns it was computed from.
+  static constexpr bool S_EARLY = D == 64;
   static constexpr int NK = D == 64 ? 3 : 2;          // K ring depth
   static constexpr int NV = D == 64 ? 3 : 2;          // V ring depth
   // byte offset, inside a tile, of the 16 columns of k-step ks of the Q K^T contraction
@@ -57,9 +57,7 @@ struct Cfg {
   static constexpr uint32_t Q = 0;
   static constexpr uint32_t K0 = Q + 2 * TILE;
   static constexpr uint32_t V0 = K0 + NK * TILE;
-  // P_SMEM only: [stream][two 64-key blocks of 128 rows x 128 B]
-  static constexpr uint32_t P0 = V0 + NV * TILE;
-  static constexpr uint32_t BAR = P0 + (P_SMEM ? 4 * BLK : 0);
+  static constexpr uint32_t BAR = V0 + NV * TILE;
   // barrier slots (8 bytes each)
   // V of tile u and K of tile u + 1 travel as a pair: they are wanted in the same iteration of the MMA warp and
   // released by it together, so one full and one empty barrier per pair (B_F, B_E) serve both; K of the first
@@ -67,12 +65,13 @@ struct Cfg {
   static_assert(NK == NV, "K and V rings advance together");
   static constexpr int NP = NV;
   static constexpr int B_Q = 0, B_K0 = 1, B_K0E = 2, B_F = 3, B_E = B_F + NP, B_SF = B_E + NP,
-                       B_PF = B_SF + 2, B_OF = B_PF + 2, B_SE = B_OF + 2 /* S read, P_SMEM only */, B_COUNT = B_SE + 2;
+                       B_PF = B_SF + 2, B_OF = B_PF + 2, B_SE = B_OF + 2 /* S read, S_EARLY only */, B_COUNT = B_SE + 2;
   static constexpr uint32_t MISC = BAR + 8 * ((B_COUNT + 7) / 8 * 8);
   static constexpr uint32_t TOTAL = MISC + 64;
   static constexpr uint32_t ALLOC = TOTAL + 1024;     // slack for manual 1024-byte alignment
   // TMEM columns
-  static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL0 = 256, O_COL1 = 384, TMEM_COLS = 512;
+  static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL0 = 256, O_COL1 = S_EARLY ? 320 : 384, TMEM_COLS = 512;
+  static constexpr uint32_t P_COL0 = S_EARLY ? 384 : S_COL0, P_COL1 = S_EARLY ? 448 : S_COL1;   // packed bf16, 64 columns
 };
 
 // The two bf16 values of a packed word, widened exactly.  The row sum is taken over these rounded weights, the
@@ -341,18 +340,12 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
                  IDESC_S, k > 0);
         tc_commit(bar(C::B_SF + j));
       };
-      const uint32_t p_lo = ((base + C::P0) >> 4) | LO_KMAJOR;
       auto issue_pv = [&](int j, int vs, bool first) {
         const uint32_t b0 = v_lo + vs * (C::TILE >> 4);
-        const uint32_t t_p = tmem_base + (j ? C::S_COL1 : C::S_COL0), t_o = tmem_base + (j ? C::O_COL1 : C::O_COL0);
+        const uint32_t t_p = tmem_base + (j ? C::P_COL1 : C::P_COL0), t_o = tmem_base + (j ? C::O_COL1 : C::O_COL0);
 #pragma unroll
-        for (int k = 0; k < BN / 16; ++k) {
-          if constexpr (C::P_SMEM)
-            mma_ss(t_o, desc(p_lo + j * ((2 * C::BLK) >> 4) + (((k >> 2) * C::BLK + (k & 3) * 32) >> 4)),
-                   desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
-          else
-            mma_ts(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
-        }
+        for (int k = 0; k < BN / 16; ++k)
+          mma_ts(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
         tc_commit(bar(C::B_OF + j));
       };
       Merge mg;
@@ -360,7 +353,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       int cur_tile, cur_uses, nxt_tile = 0, nxt_uses = 0;
       bool has_cur = mg.next(L, cur_tile, cur_uses);
       int pv_cnt[2] = {0, 0};
-      int s_cnt[2] = {0, 0};   // P_SMEM: S tiles issued per stream
+      int s_cnt[2] = {0, 0};   // S_EARLY: S tiles issued per stream
       mbar_wait(bar(C::B_Q), 0, wc);
       if (has_cur) {
         mbar_wait(bar(C::B_K0), 0, wc);
@@ -375,7 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         // the TMA barrier first (V of this tile and K of the next): the data has normally landed long ago, and
         // checking here keeps it out of the gap between a stream's P arriving and its MMAs being issued
         mbar_wait(bar(C::B_F + vs), (u / C::NP) & 1, wc);
-        if constexpr (C::P_SMEM) {
+        if constexpr (C::S_EARLY) {
           // the next tile's scores first: S is free as soon as the softmax warps have read the current one
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
@@ -436,8 +429,8 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       const int u0 = (int)(entry & ~RF_PARTIAL_BIT) * BN;
       mbar_wait(bar(C::B_SF + j), it & 1, wc);
       tc_fence_after();
-      if constexpr (C::P_SMEM) {
-        // S into registers and the accumulator handed back at once; the exponentials go to shared memory.
+      if constexpr (C::S_EARLY) {
+        // S into registers and the accumulator handed back at once; P goes to TMEM columns of its own.
         uint32_t s[128];
         {
           uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
@@ -479,7 +472,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           l_exact *= alpha;
         }
         if (it > 0) {
-          // P V of the previous tile reads the shared-memory P this tile is about to overwrite, and O may
+          // P V of the previous tile reads the P columns this tile is about to overwrite, and O may
           // only be rescaled once everything issued into it has landed.  Waiting here also keeps this stream
           // at most one tile ahead of the MMA warp, which tracks the P barrier by phase parity.
           mbar_wait(bar(C::B_OF + j), (it - 1) & 1, wc);
@@ -501,27 +494,29 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         const float m_use = m_run == -INFINITY ? 0.f : m_run;
         const float2 sc2 = make_float2(sc, sc), mneg = make_float2(-m_use, -m_use);
         float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
-        const uint32_t p_row = base + C::P0 + j * 2 * C::BLK + row_in_tile * 128;
+        uint32_t pk[64];
 #pragma unroll
-        for (int c = 0; c < 128; c += 8) {
-          uint32_t pw[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            float2 e = __ffma2_rn(make_float2(__uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1])), sc2, mneg);
-            e.x = ex2(e.x);
-            e.y = ex2(e.y);
-            pw[i] = pack_bf16(e.x, e.y);
-            la = __fadd2_rn(la, e);
-            lb = __fadd2_rn(lb, unpack_bf16(pw[i]));
-          }
-          // 8 keys = one 16-byte chunk of the row; 128-byte swizzle: chunk index XOR (row mod 8)
-          const uint32_t chunk = (uint32_t)((c >> 3) & 7) ^ (uint32_t)(row_in_tile & 7);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_row + (c >> 6) * C::BLK + (chunk << 4)),
-                       "r"(pw[0]), "r"(pw[1]), "r"(pw[2]), "r"(pw[3]) : "memory");
+        for (int c = 0; c < 128; c += 4) {
+          float2 e0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, mneg);
+          float2 e1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, mneg);
+          e0.x = ex2(e0.x); e0.y = ex2(e0.y);
+          e1.x = ex2(e1.x); e1.y = ex2(e1.y);
+          pk[c / 2] = pack_bf16(e0.x, e0.y);
+          pk[c / 2 + 1] = pack_bf16(e1.x, e1.y);
+          la = __fadd2_rn(la, __fadd2_rn(e0, e1));
+          lb = __fadd2_rn(lb, __fadd2_rn(unpack_bf16(pk[c / 2]), unpack_bf16(pk[c / 2 + 1])));
         }
         l_exact += la.x + la.y;
         l_run += lb.x + lb.y;
-        fence_proxy_async_smem();
+        {
+          const uint32_t t_p = tmem_base + lane_sel + (j ? C::P_COL1 : C::P_COL0);
+          uint32_t(&p0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[0]);
+          uint32_t(&p1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[32]);
+          tmem_st32(t_p, p0);
+          tmem_st32(t_p + 32, p1);
+          tc_wait_st();
+        }
+        tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(C::B_PF + j));
         continue;

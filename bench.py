@@ -31,7 +31,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one rf_attn_kernel launch, from single-pass ncu captures
 # (profiles/rf_attn_kernel_hunyuan720p_dram_bytes.md); None where no capture exists.
-ATTN_DRAM_BYTES = {"hunyuan720p": 4.21e9, "sweep_33x3600": 4.21e9, "sweep_16x2040": 0.733e9}
+ATTN_DRAM_BYTES = {"hunyuan720p": 4.69e9, "sweep_33x3600": 4.69e9, "sweep_16x2040": 0.734e9}
 
 
 def peaks():

@@ -68,6 +68,9 @@ typedef struct {
   float   alpha;            /* recall threshold of Algorithm 1, in (0, 1] */
   int32_t block_m, block_n; /* tile of the block mask: query rows x key slots */
   int32_t temporal_permute; /* 1: Temporal heads run in position-major token order (slot = pos*T + frame) */
+  int32_t two_mask;         /* 0: Algorithm 1 as printed (Spatial, Temporal, else Textural).  1: the ablation of
+                               Sec. 4.4 / Table 2 with only the Spatial and Temporal masks: a head that reaches alpha
+                               with neither takes the one of larger recall (Temporal on equality), never Textural */
 } rf_params;
 
 /*

@@ -150,24 +150,32 @@ def recall(P: np.ndarray, kept: np.ndarray) -> float:
     return float((P * kept).sum(axis=1).mean())
 
 
-def decide(R_temporal: float, R_spatial: float, alpha: float) -> int:
-    """Algorithm 1's branch: Temporal has priority, then Spatial, else Textural."""
+def decide(R_temporal: float, R_spatial: float, alpha: float, two_mask: bool = False) -> int:
+    """Algorithm 1's branch: Temporal has priority, then Spatial, else Textural.
+    two_mask: the ablation of Sec. 4.4 (Table 2, rows without Te) that uses only the Spatial and the
+    Temporal mask; the paper does not say what a head reaching alpha with neither gets: here the mask of
+    larger recall, Temporal on equality."""
     if R_temporal >= alpha:
         return TEMPORAL
     if R_spatial >= alpha:
         return SPATIAL
+    if two_mask:
+        return TEMPORAL if R_temporal >= R_spatial else SPATIAL
     return TEXTURAL
 
 
-def decision_margin(R_temporal: float, R_spatial: float, alpha: float) -> float:
-    """Distance of the deciding recall(s) from the threshold."""
+def decision_margin(R_temporal: float, R_spatial: float, alpha: float, two_mask: bool = False) -> float:
+    """Distance of the deciding recall(s) from the threshold (and from each other, where that decides)."""
     if R_temporal >= alpha:
         return abs(R_temporal - alpha)
-    return min(abs(R_temporal - alpha), abs(R_spatial - alpha))
+    m = min(abs(R_temporal - alpha), abs(R_spatial - alpha))
+    if two_mask and R_spatial < alpha:
+        m = min(m, abs(R_temporal - R_spatial))
+    return m
 
 
 def arm_head(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, pp: PatternParams,
-             sample_mode: int, omega: int, alpha: float):
+             sample_mode: int, omega: int, alpha: float, two_mask: bool = False):
     """ARM for one head.  q_bits, k_bits: [N, D] bf16 bit patterns.
     Returns (class, (R_temporal, R_spatial, R_textural), margin)."""
     I_glb = global_sample(g, omega)
@@ -182,11 +190,11 @@ def arm_head(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, pp: PatternPar
         R_t = recall(P_glb, keep_mask(TEMPORAL, I_glb, I_glb, g, pp))
     else:
         raise ValueError(sample_mode)
-    return decide(R_t, R_s, alpha), (R_t, R_s, R_te), decision_margin(R_t, R_s, alpha)
+    return decide(R_t, R_s, alpha, two_mask), (R_t, R_s, R_te), decision_margin(R_t, R_s, alpha, two_mask)
 
 
 def arm_classify(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, pp: PatternParams,
-                 sample_mode: int, omega: int, alpha: float):
+                 sample_mode: int, omega: int, alpha: float, two_mask: bool = False):
     """ARM over [B, H, N, D] inputs.  Returns (class int32 [B,H], recall f64 [B,H,3], margin f64 [B,H])."""
     B, H = q_bits.shape[:2]
     cls = np.zeros((B, H), dtype=np.int32)
@@ -194,7 +202,7 @@ def arm_classify(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, pp: Patter
     mar = np.zeros((B, H), dtype=np.float64)
     for b in range(B):
         for h in range(H):
-            c, r, m = arm_head(q_bits[b, h], k_bits[b, h], g, pp, sample_mode, omega, alpha)
+            c, r, m = arm_head(q_bits[b, h], k_bits[b, h], g, pp, sample_mode, omega, alpha, two_mask)
             cls[b, h], rec[b, h], mar[b, h] = c, r, m
     return cls, rec, mar
 
@@ -208,19 +216,24 @@ def windows_of(bandwidth: float, g: Geometry) -> Tuple[int, int]:
     return int(math.floor(bandwidth * g.T)), int(math.floor(bandwidth * g.S))
 
 
-def decide_plus(R_temporal: Sequence[float], R_spatial: Sequence[float], alpha: float) -> Tuple[int, int]:
+def decide_plus(R_temporal: Sequence[float], R_spatial: Sequence[float], alpha: float,
+                two_mask: bool = False) -> Tuple[int, int]:
     """Recalls per candidate bandwidth (ascending).  The pattern is chosen as in Algorithm 1 (Temporal
     first, then Spatial, else Textural), a pattern qualifying if ANY candidate reaches alpha; its
-    bandwidth is the smallest candidate that does.  Returns (class, candidate index or -1)."""
+    bandwidth is the smallest candidate that does.  Returns (class, candidate index or -1).
+    two_mask (see decide): if nothing qualifies, the mask of larger recall at the widest candidate."""
     for cls, R in ((TEMPORAL, R_temporal), (SPATIAL, R_spatial)):
         for i, r in enumerate(R):
             if r >= alpha:
                 return cls, i
+    if two_mask:
+        last = len(R_temporal) - 1
+        return (TEMPORAL if R_temporal[last] >= R_spatial[last] else SPATIAL), last
     return TEXTURAL, -1
 
 
 def arm_head_plus(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, bandwidths: Sequence[float], tau: int,
-                  sample_mode: int, omega: int, alpha: float):
+                  sample_mode: int, omega: int, alpha: float, two_mask: bool = False):
     """ARM with dynamic bandwidth for one head: every candidate bandwidth's Temporal and Spatial recall on
     the same approximate scores, then decide_plus.  Returns (class, index, window, R_t list, R_s list),
     window = w_s of the chosen bandwidth for Temporal, w_f for Spatial, -1 for Textural."""
@@ -237,7 +250,7 @@ def arm_head_plus(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, bandwidth
         pp = PatternParams(wf, ws, tau)
         R_t.append(recall(P_t, keep_mask(TEMPORAL, I_t, I_t, g, pp)))
         R_s.append(recall(P_glb, keep_mask(SPATIAL, I_glb, I_glb, g, pp)))
-    cls, idx = decide_plus(R_t, R_s, alpha)
+    cls, idx = decide_plus(R_t, R_s, alpha, two_mask)
     window = -1
     if cls == TEMPORAL:
         window = windows_of(bandwidths[idx], g)[1]

@@ -28,6 +28,7 @@ rf_status check_params(const rf_params* p) {
   if (!(p->alpha > 0.f && p->alpha <= 1.f)) return RF_ERR_INVALID_ARG;
   if (!pow2(p->block_m) || !pow2(p->block_n) || p->block_m < 16 || p->block_n < 16) return RF_ERR_INVALID_ARG;
   if (p->temporal_permute != 0 && p->temporal_permute != 1) return RF_ERR_INVALID_ARG;
+  if (p->two_mask != 0 && p->two_mask != 1) return RF_ERR_INVALID_ARG;
   return RF_OK;
 }
 
@@ -54,10 +55,13 @@ RfGeom make_geom(const rf_shape* s, int wf, int ws, int tau, int bm, int bn, int
   g.nQ = rf_cdiv(g.N, bm);
   g.nKmax = rf_cdiv(g.N, bn);
   g.permute = permute;
+  g.two_mask = 0;
   return g;
 }
 RfGeom make_geom(const rf_shape* s, const rf_params* p) {
-  return make_geom(s, p->frame_window, p->spatial_window, p->textural_stride, p->block_m, p->block_n, p->temporal_permute);
+  RfGeom g = make_geom(s, p->frame_window, p->spatial_window, p->textural_stride, p->block_m, p->block_n, p->temporal_permute);
+  g.two_mask = p->two_mask;
+  return g;
 }
 
 size_t tensor_bytes(const RfGeom& g) { return align_up((size_t)g.B * g.H * g.N * g.D * sizeof(__nv_bfloat16)); }

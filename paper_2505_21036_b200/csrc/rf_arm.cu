@@ -349,7 +349,7 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
 //   dynamic bandwidth: a pattern qualifies if any candidate window reaches alpha, Temporal before Spatial;
 //   the head takes the smallest qualifying window (candidates ascend); Textural heads get window -1.
 __global__ void __launch_bounds__(256) rf_arm_decide_kernel(int nb, int nb_user, int n_loc, int n_glb, int n_pad, int sample_mode,
-                                                             float alpha, ArmWindows win, int with_tex,
+                                                             float alpha, int two_mask, ArmWindows win, int with_tex,
                                                              const float* __restrict__ rows_loc,
                                                              const float* __restrict__ rows_glb,
                                                              int32_t* __restrict__ head_class,
@@ -382,9 +382,16 @@ __global__ void __launch_bounds__(256) rf_arm_decide_kernel(int nb, int nb_user,
     if (head_window == nullptr) {
       const float Rt = R[0], Rs = R[nb], Rc = R[2 * nb];
       if (recall) { recall[bh * 3] = Rt; recall[bh * 3 + 1] = Rs; recall[bh * 3 + 2] = Rc; }
-      head_class[bh] = Rt >= alpha ? RF_TEMPORAL : (Rs >= alpha ? RF_SPATIAL : RF_TEXTURAL);
+      // Algorithm 1; with only two masks (ablation) a head that reaches alpha with neither takes the larger recall
+      const int otherwise = two_mask ? (Rt >= Rs ? RF_TEMPORAL : RF_SPATIAL) : RF_TEXTURAL;
+      head_class[bh] = Rt >= alpha ? RF_TEMPORAL : (Rs >= alpha ? RF_SPATIAL : otherwise);
     } else {
       int cls = RF_TEXTURAL, window = -1;
+      if (two_mask) {   // nothing qualifies: the larger recall at the widest candidate, with that bandwidth
+        const bool t = R[nb_user - 1] >= R[nb + nb_user - 1];
+        cls = t ? RF_TEMPORAL : RF_SPATIAL;
+        window = t ? win.ws[nb_user - 1] : win.wf[nb_user - 1];
+      }
       // nb slots were evaluated (the caller's nb_user candidates, padded by repeating the last one)
       for (int i = nb_user - 1; i >= 0; --i)
         if (R[nb + i] >= alpha) { cls = RF_SPATIAL; window = win.wf[i]; }
@@ -477,7 +484,7 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
     default: e = cudaErrorInvalidValue;
   }
   if (e != cudaSuccess) return e;
-  rf_arm_decide_kernel<<<heads, 256, 0, st>>>(NB, nb, n_loc, n_glb, n_pad, sample_mode, alpha, win, tex ? 1 : 0, rows_loc,
+  rf_arm_decide_kernel<<<heads, 256, 0, st>>>(NB, nb, n_loc, n_glb, n_pad, sample_mode, alpha, g.two_mask, win, tex ? 1 : 0, rows_loc,
                                               rows_glb, head_class, head_window, recall, recall_plus);
   return cudaGetLastError();
 }

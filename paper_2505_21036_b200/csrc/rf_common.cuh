@@ -20,6 +20,7 @@ struct RfGeom {
   int LkvTex;            // key slots of a Textural head: T*nC + L
   int BM, BN, nQ, nKmax; // block mask tile and its extents
   int permute;           // Temporal heads in position-major order
+  int two_mask;          // ARM decides between Spatial and Temporal only (ablation of Sec. 4.4)
 };
 
 // Device-side error reporting: first error wins, kernels never trap.

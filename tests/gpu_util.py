@@ -33,12 +33,12 @@ def bits_of(t: torch.Tensor) -> np.ndarray:
 class Run:
     """One workload resident on the GPU with its schedule and workspace."""
 
-    def __init__(self, wl, qkv=None, block=128, temporal_permute=1):
+    def __init__(self, wl, qkv=None, block=128, temporal_permute=1, two_mask=0):
         self.wl = wl
         self.q_bits, self.k_bits, self.v_bits = qkv if qkv is not None else synth.make_qkv(wl)
         self.q, self.k, self.v = (to_dev(x) for x in (self.q_bits, self.k_bits, self.v_bits))
         self.shape = api.shape_of(wl)
-        self.params = api.params_of(wl, block, block, temporal_permute)
+        self.params = api.params_of(wl, block, block, temporal_permute, two_mask)
         self.ws = api.alloc_workspace(self.shape, self.params, "cuda")
         self.sched = api.Schedule(self.shape, self.params, "cuda", with_bitmap=True)
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")

@@ -91,6 +91,35 @@ def test_arm_mid(D, mode):
     check_arm(wl)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_arm_two_mask_ablation(mode):
+    """Only the Spatial and Temporal masks (Table 2, rows without Te): weakly planted heads reach alpha with
+    neither and must take the mask of larger recall; strongly planted ones decide as in Algorithm 1."""
+    for amp in (0.5, 1.5):
+        wl = synth.small_workload("two_mask", H=6, D=64, T=6, fh=12, fw=11, L=37, wf=1, ws=20, tau=2, mode=mode, omega=6,
+                                  amp=amp)
+        run = gu.Run(wl, two_mask=1)
+        cls_gpu, rec_gpu = run.arm()
+        cls_ref, rec_ref, margin = orc.arm_classify(run.q_bits, run.k_bits, gu.geom(wl), gu.pparams(wl), wl.sample_mode,
+                                                    wl.sample_stride, wl.alpha, two_mask=True)
+        assert np.abs(rec_gpu - rec_ref).max() <= gu.RECALL_ABS
+        assert not (cls_gpu == X_).any() and not (cls_ref == X_).any()
+        decided = margin > gu.TIE_MARGIN
+        assert decided.sum() >= 4
+        assert np.array_equal(cls_gpu[decided], cls_ref[decided])
+        three = orc.arm_classify(run.q_bits, run.k_bits, gu.geom(wl), gu.pparams(wl), wl.sample_mode, wl.sample_stride,
+                                 wl.alpha)[0]
+        if amp == 0.5:
+            assert (three == X_).any()          # the ablation really changes something here
+        # the pipeline runs on whatever the ablation picked
+        run.build()
+        O, lse = run.sparse()
+        for h in (0, 3):
+            Or, lr = orc.masked_attention(run.q_bits[0, h], run.k_bits[0, h], run.v_bits[0, h], int(cls_gpu[0, h]),
+                                          gu.geom(wl), gu.pparams(wl))
+            gu.check_attention(O[0, h], lse[0, h], Or, lr, f"two-mask head {h}", strict=False)
+
+
 def test_arm_is_deterministic():
     wl = mid_workload()
     run = gu.Run(wl)

@@ -82,6 +82,32 @@ def test_dynamic_bandwidth_pipeline(mode):
         gu.check_attention(O[h], LSE[h], Or, lr, f"plus head {h} class {cls} window {w}", strict=False)
 
 
+def test_dynamic_bandwidth_with_two_masks():
+    """Dynamic bandwidth without the Textural mask: a head no candidate qualifies for takes the mask of larger
+    recall at the widest candidate."""
+    wl = synth.small_workload("plus2", H=4, D=64, T=8, fh=16, fw=16, L=32, tau=2, mode=0, omega=4, amp=2.0)
+    heads = [planted_groups(wl, 0, frames_per_group=1), planted_groups(wl, 2, positions_per_group=16),
+             synth.make_head(wl, 0, 4, kind="lowrank"), synth.make_head(wl, 0, 5, kind="none")]
+    q, k, v = (np.stack([h[i] for h in heads])[None] for i in range(3))
+    run = gu.Run(wl, qkv=(q, k, v), two_mask=1)
+    head_window = torch.full((wl.B, wl.H), -7, dtype=torch.int32, device="cuda")
+    rec = torch.zeros((wl.B, wl.H, 2, len(BWS)), dtype=torch.float32, device="cuda")
+    api.rf_arm_classify_plus(run.shape, run.params, BWS, run.q, run.k, run.head_class, head_window, rec, run.ws)
+    torch.cuda.synchronize()
+    cls_gpu, win_gpu = run.head_class.cpu().numpy()[0], head_window.cpu().numpy()[0]
+    g = gu.geom(wl)
+    fell_back = 0
+    for h in range(wl.H):
+        cls, idx, window, Rt, Rs = orc.arm_head_plus(q[0, h], k[0, h], g, BWS, wl.textural_stride, 0, wl.sample_stride,
+                                                     wl.alpha, two_mask=True)
+        assert cls in (orc.SPATIAL, orc.TEMPORAL) and window >= 0
+        margin = min([abs(r - wl.alpha) for r in list(Rt) + list(Rs)] + [abs(Rt[-1] - Rs[-1])])
+        if margin > gu.TIE_MARGIN:
+            assert (int(cls_gpu[h]), int(win_gpu[h])) == (cls, window), h
+        fell_back += max(max(Rt), max(Rs)) < wl.alpha
+    assert fell_back >= 1
+
+
 def test_plus_entry_points_with_null_windows_equal_the_plain_ones():
     wl = synth.WORKLOADS["tiny"]
     run = gu.Run(wl)

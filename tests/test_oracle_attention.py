@@ -202,6 +202,27 @@ def test_algorithm1_truth_table(Rt, Rs, expect):
     assert orc.decide(Rt, Rs, 0.9) == expect
 
 
+def test_two_mask_ablation_never_picks_textural_and_agrees_with_algorithm1_elsewhere():
+    """Table 2's rows without the Textural mask: same decision wherever Algorithm 1 picks Spatial or Temporal,
+    the mask of larger recall (Temporal on equality) where it would have picked Textural."""
+    grid = [i / 20.0 for i in range(21)]
+    for alpha in (0.5, 0.9, 1.0):
+        for Rt in grid:
+            for Rs in grid:
+                three, two = orc.decide(Rt, Rs, alpha), orc.decide(Rt, Rs, alpha, two_mask=True)
+                assert two in (TEMPORAL, SPATIAL)
+                if three != TEXTURAL:
+                    assert two == three
+                else:
+                    assert two == (TEMPORAL if Rt >= Rs else SPATIAL)
+    assert orc.decide_plus([0.1, 0.2, 0.3], [0.2, 0.3, 0.25], 0.9, two_mask=True) == (TEMPORAL, 2)
+    assert orc.decide_plus([0.1, 0.2, 0.3], [0.2, 0.3, 0.35], 0.9, two_mask=True) == (SPATIAL, 2)
+    assert orc.decide_plus([0.1, 0.95, 0.99], [0.2, 0.3, 0.35], 0.9, two_mask=True) == (TEMPORAL, 1)
+    assert orc.decide_plus([0.1, 0.2, 0.3], [0.2, 0.3, 0.35], 0.9) == (TEXTURAL, -1)
+    assert orc.decision_margin(0.5, 0.52, 0.9, two_mask=True) == pytest.approx(0.02)
+    assert orc.decision_margin(0.5, 0.93, 0.9, two_mask=True) == pytest.approx(0.03)
+
+
 def test_margin():
     assert orc.decision_margin(0.95, 0.2, 0.9) == pytest.approx(0.05)
     assert orc.decision_margin(0.5, 0.93, 0.9) == pytest.approx(0.03)

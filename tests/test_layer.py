@@ -67,3 +67,24 @@ def test_layer_equals_the_entry_points_and_graph_replay_equals_eager(plus):
     assert len(graphed._graphs) == 1
     eager.check()
     graphed.check()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("groups", [1, 2, 4])
+def test_host_staged_call_equals_the_resident_pipeline(groups):
+    wl, eager = make_layer("cuda", dense_fraction=0.0)
+    from paper_2505_21036_b200.layer import HostStagedAttention
+    staged = HostStagedAttention(api.shape_of(wl), api.params_of(wl), "cuda", groups=groups)
+    host = [torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in synth.make_qkv(wl)]
+    oh = torch.full(host[0].shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+    for _ in range(2):                                   # back-to-back calls reuse the staging buffers
+        staged(*host, oh)
+    torch.cuda.synchronize()
+    q, k, v = (t.cuda() for t in host)
+    o = torch.empty_like(q)
+    eager(q, k, v, o, None, step=0, num_steps=1)
+    torch.cuda.synchronize()
+    assert int(staged.status.item()) == 0
+    assert torch.equal(oh.view(torch.int16), o.cpu().view(torch.int16))
+    with pytest.raises(ValueError):
+        HostStagedAttention(api.shape_of(wl), api.params_of(wl), "cuda", groups=3)

@@ -38,8 +38,8 @@ template <int D>
 struct Cfg {
   static constexpr int KB = (D + 63) / 64;            // 64-column (128-byte) blocks per row
   // first column of the second block.  D = 96 is fetched as columns [0,64) and [64,128): the TMA box
-  // reaches past the tensor's 96 columns and the missing ones arrive as zeros, so that P V can run as
-  // one N = 128 MMA per k-step (the 32 extra accumulator columns stay zero and are never stored)
+  // reaches past the tensor's 96 columns and the missing ones arrive as zeros; they are never read
+  // (Q K^T runs 6 k-steps, P V is one N = 96 MMA per k-step over one and a half 64-column blocks)
   static constexpr int COL1 = 64;
   static constexpr uint32_t BLK = 128 * 128;          // bytes of one 128-row x 64-col bf16 block
   static constexpr uint32_t TILE = KB * BLK;          // bytes of one 128-row tile
@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   using C = Cfg<D>;
   constexpr int KB = C::KB;
   constexpr uint32_t IDESC_S = idesc_bf16(BM, BN, 0);
-  constexpr uint32_t IDESC_PV = idesc_bf16(BM, D == 96 ? 128 : D, 1);
+  constexpr uint32_t IDESC_PV = idesc_bf16(BM, D, 1);
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;

@@ -16,8 +16,8 @@ Readings taken where the paper is silent (each also listed in the design notes):
   * tokens: frame-major, row-major inside a frame, text tokens appended last;
   * Spatial head keeps |frame(i) - frame(j)| <= w_f (Eq. 3: the significant frames
     of frame f are its neighbours); Temporal head keeps |pos(i) - pos(j)| <= w_s with
-    pos the flattened in-frame index (Sec. 3.2, "locality within a single-frame
-    sub-sequence"); text rows and text columns are always kept for both;
+    pos the flattened in-frame index (Sec. 3.2 describes Temporal heads as local inside one
+    frame's sub-sequence and periodic across frames); text rows and text columns are always kept for both;
   * Textural head keeps key/value token (y, x) of every frame iff y mod tau == x mod tau
     (Eq. 4), plus all text keys, for every query (Eq. 5: all-zero mask on K_C, V_C);
   * recall (Eq. 6) is the share of a row's unmasked softmax mass that falls on kept

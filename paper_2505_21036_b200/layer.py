@@ -3,8 +3,8 @@
 Policy only: which entry points of the C ABI run at which denoising step, with which buffers.  Every
 arithmetic step is a kernel of the library.
 
-  * the first `dense_fraction` of the sampling steps run dense attention (Sec. 4.2: "we keep the first 10%
-    timesteps using dense calculation");
+  * the first `dense_fraction` of the sampling steps run dense attention (Sec. 4.2 keeps the first tenth of
+    the timesteps dense);
   * every later step runs ARM -> tile schedule -> pattern-masked attention (Fig. 2a: the head categories are
     determined online, per call);
   * with `graph=True` the three calls of a sparse step are captured once into a CUDA graph per set of

@@ -16,7 +16,7 @@ def test_dense_step_policy_and_speedup_arithmetic():
     wl, layer = make_layer("cpu")
     assert layer.dense_steps(50) == 5 and layer.dense_steps(10) == 1 and layer.dense_steps(4) == 1
     assert [layer.is_dense_step(s, 50) for s in (0, 4, 5, 49)] == [True, True, False, False]
-    # Sec. 4.2: 50 % sparsity with the first 10 % of the steps dense is quoted as "about 1.85x"
+    # Sec. 4.2: 50 % sparsity with the first tenth of the steps dense; the paper's attention speed-up figure is 1.85x
     assert layer.expected_attention_speedup(50, 0.5) == pytest.approx(1.0 / (0.1 + 0.9 * 0.5))
     assert 1.8 < layer.expected_attention_speedup(50, 0.5) < 1.86
     wl, none_dense = make_layer("cpu", dense_fraction=0.0)

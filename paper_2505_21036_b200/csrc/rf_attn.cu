@@ -369,7 +369,10 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         // checking here keeps it out of the gap between a stream's P arriving and its MMAs being issued
         mbar_wait(bar(C::B_F + vs), (u / C::NP) & 1, wc);
         if constexpr (C::S_EARLY) {
-          // the next tile's scores first: S is free as soon as the softmax warps have read the current one
+          // Per stream: the next tile's scores (S is free as soon as the softmax warps have read the current
+          // one), then O += P V of the current tile.  Stream 1's next scores are thus only issued once stream 0
+          // has delivered its P: the two streams settle half a tile apart and take turns at the MUFU unit
+          // instead of sitting in their exponentials at the same time.
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             if (has_nxt && (nxt_uses & (1 << j))) {
@@ -378,9 +381,6 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
               issue_s(j, ksn);
               ++s_cnt[j];
             }
-          }
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
             if (cur_uses & (1 << j)) {
               mbar_wait(bar(C::B_PF + j), pv_cnt[j] & 1, wc);
               tc_fence_after();
@@ -471,12 +471,15 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           l_run *= alpha;
           l_exact *= alpha;
         }
-        if (it > 0) {
-          // P V of the previous tile reads the P columns this tile is about to overwrite, and O may
-          // only be rescaled once everything issued into it has landed.  Waiting here also keeps this stream
-          // at most one tile ahead of the MMA warp, which tracks the P barrier by phase parity.
+        // P V of the previous tile reads the P columns this tile is about to overwrite, and O may only be
+        // rescaled once everything issued into it has landed.  The wait sits in front of the P store (the
+        // exponentials of this tile run under the previous tile's P V); it also keeps this stream at most
+        // one tile ahead of the MMA warp, which tracks the P barrier by phase parity.
+        bool o_landed = it == 0;
+        if (it > 0 && any_raise) {
           mbar_wait(bar(C::B_OF + j), (it - 1) & 1, wc);
-          if (any_raise) {
+          o_landed = true;
+          {
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
@@ -508,6 +511,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         }
         l_exact += la.x + la.y;
         l_run += lb.x + lb.y;
+        if (!o_landed) mbar_wait(bar(C::B_OF + j), (it - 1) & 1, wc);
         {
           const uint32_t t_p = tmem_base + lane_sel + (j ? C::P_COL1 : C::P_COL0);
           uint32_t(&p0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&pk[0]);

@@ -107,7 +107,8 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
   const bool stream1 = qt0 + 1 < nt;
   const CUtensorMap* map_q = &maps.q[which];
   const CUtensorMap* map_k = &maps.k[which];
-  const bool t_generic = sm.want_t && stride != 1;    // needs per-key positions
+  // positions equal sample indices only while the sample is contiguous and stays inside the first frame
+  const bool t_generic = sm.want_t && (stride != 1 || n > g.S);    // needs per-key positions
 
   if (tid == 0) {
     mbar_init(bar(C::B_Q), 1);

@@ -15,16 +15,17 @@ import gpu_util as gu
 pytestmark = pytest.mark.gpu
 
 
-def draw_case(seed):
-    rng = np.random.default_rng(9000 + seed)
+def draw_case(seed, large=False):
+    rng = np.random.default_rng((77000 if large else 9000) + seed)
     D = int(rng.choice([64, 96, 128]))
-    T = int(rng.integers(1, 8))
-    fh, fw = int(rng.integers(1, 13)), int(rng.integers(1, 13))
+    T = int(rng.integers(1, 14 if large else 8))
+    hi = 21 if large else 13
+    fh, fw = int(rng.integers(1, hi)), int(rng.integers(1, hi))
     S = fh * fw
     L = int(rng.choice([0, 1, 17, 130]))
     if T * S + L < 2:
         L = 17
-    kw = dict(B=int(rng.choice([1, 2])), H=4, D=D, T=T, fh=fh, fw=fw, L=L,
+    kw = dict(B=1 if large else int(rng.choice([1, 2])), H=4, D=D, T=T, fh=fh, fw=fw, L=L,
               wf=int(rng.integers(0, T + 1)), ws=int(rng.integers(0, S + 1)), tau=int(rng.integers(1, 5)),
               mode=int(rng.integers(0, 2)), omega=int(rng.integers(1, max(2, S // 2 + 1))),
               amp=float(rng.choice([0.0, 0.8, 1.5, 2.5])))
@@ -35,9 +36,18 @@ def draw_case(seed):
     return wl, permute, two_mask, classes
 
 
-@pytest.mark.parametrize("seed", range(32))
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("RF_FUZZ_FROM", "0")), int(__import__("os").environ.get("RF_FUZZ_TO", "32"))))
 def test_random_case(seed):
-    wl, permute, two_mask, classes = draw_case(seed)
+    check_case(seed, *draw_case(seed))
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("RF_FUZZ_LARGE_FROM", "0")),
+                                       int(__import__("os").environ.get("RF_FUZZ_LARGE_TO", "8"))))
+def test_random_case_up_to_forty_tiles(seed):
+    check_case(seed, *draw_case(seed, large=True))
+
+
+def check_case(seed, wl, permute, two_mask, classes):
     g, pp = gu.geom(wl), gu.pparams(wl)
     run = gu.Run(wl, temporal_permute=permute, two_mask=two_mask)
     # ARM
@@ -63,3 +73,49 @@ def test_random_case(seed):
         Od, lsed = run.dense()
         Or, lr = orc.masked_attention(run.q_bits[0, 1], run.k_bits[0, 1], run.v_bits[0, 1], orc.DENSE, g, pp)
         gu.check_attention(Od[0, 1], lsed[0, 1], Or, lr, f"fuzz {seed} dense", strict=False)
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("RF_FUZZ_PLUS_FROM", "0")),
+                                       int(__import__("os").environ.get("RF_FUZZ_PLUS_TO", "12"))))
+def test_random_case_dynamic_bandwidth(seed):
+    """The dynamic-bandwidth variant on drawn shapes: candidate lists of one to four bandwidths, the per-head
+    window ARM picks, the schedule and the attention that honour it."""
+    import torch
+    from paper_2505_21036_b200 import api
+    wl, permute, two_mask, _ = draw_case(seed)
+    rng = np.random.default_rng(555 + seed)
+    bws = sorted(set(float(x) for x in rng.choice([0.05, 0.125, 0.2, 0.25, 0.4, 0.5, 0.75, 1.0], size=int(rng.integers(1, 5)))))
+    g = gu.geom(wl)
+    run = gu.Run(wl, temporal_permute=permute, two_mask=two_mask)
+    head_window = torch.full((wl.B, wl.H), -7, dtype=torch.int32, device="cuda")
+    rec = torch.zeros((wl.B, wl.H, 2, len(bws)), dtype=torch.float32, device="cuda")
+    api.rf_arm_classify_plus(run.shape, run.params, bws, run.q, run.k, run.head_class, head_window, rec, run.ws)
+    torch.cuda.synchronize()
+    cls_gpu, win_gpu, rec_gpu = run.head_class.cpu().numpy(), head_window.cpu().numpy(), rec.cpu().numpy()
+    for b in range(wl.B):
+        for h in range(wl.H):
+            cls, idx, window, Rt, Rs = orc.arm_head_plus(run.q_bits[b, h], run.k_bits[b, h], g, bws, wl.textural_stride,
+                                                         wl.sample_mode, wl.sample_stride, wl.alpha, two_mask=bool(two_mask))
+            assert np.abs(rec_gpu[b, h, 0] - np.asarray(Rt)).max() <= gu.RECALL_ABS, (seed, b, h)
+            assert np.abs(rec_gpu[b, h, 1] - np.asarray(Rs)).max() <= gu.RECALL_ABS, (seed, b, h)
+            margin = min([abs(r - wl.alpha) for r in list(Rt) + list(Rs)] + ([abs(Rt[-1] - Rs[-1])] if two_mask else []))
+            if margin > gu.TIE_MARGIN:
+                assert (int(cls_gpu[b, h]), int(win_gpu[b, h])) == (cls, window), (seed, b, h)
+    api.rf_build_block_mask_plus(run.shape, run.params, run.head_class, head_window, run.sched, run.status)
+    o = torch.full((wl.B, wl.H, wl.N, wl.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((wl.B, wl.H, wl.N), float("nan"), dtype=torch.float32, device="cuda")
+    api.rf_sparse_attn_fwd_plus(run.shape, run.params, run.q, run.k, run.v, run.head_class, head_window, run.sched, o, lse,
+                                run.ws, run.status)
+    torch.cuda.synchronize()
+    assert int(run.status.item()) == 0
+    O, LSE = o.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
+    for b in range(wl.B):
+        for h in range(wl.H):
+            cls, w = int(cls_gpu[b, h]), int(win_gpu[b, h])
+            pp = orc.PatternParams(w if cls == orc.SPATIAL else wl.frame_window,
+                                   w if cls == orc.TEMPORAL else wl.spatial_window, wl.textural_stride)
+            got = run.lists(b, h)
+            for a in range(run.sched.nQ):
+                assert got[a] == orc.tile_row(cls, g, pp, bool(permute), 128, 128, a), (seed, b, h, a)
+            Or, lr = orc.masked_attention(run.q_bits[b, h], run.k_bits[b, h], run.v_bits[b, h], cls, g, pp)
+            gu.check_attention(O[b, h], LSE[b, h], Or, lr, f"fuzz+ {seed} b{b} h{h} class {cls} window {w}", strict=False)

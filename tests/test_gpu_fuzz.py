@@ -69,6 +69,15 @@ def check_case(seed, wl, permute, two_mask, classes):
             assert int(run.sched.kv_len[b, h]) == orc.kv_len(cls, g, pp)
             Or, lr = orc.masked_attention(run.q_bits[b, h], run.k_bits[b, h], run.v_bits[b, h], cls, g, pp)
             gu.check_attention(O[b, h], lse[b, h], Or, lr, f"fuzz {seed} b{b} h{h} class {cls}", strict=False)
+    # the schedule builder alone at a smaller tile (the attention kernel itself only takes 128 x 128)
+    block = (16, 32, 64)[seed % 3]
+    small = gu.Run(wl, block=block, temporal_permute=permute)
+    small.force_classes(classes)
+    small.build()
+    for b in range(wl.B):
+        for h in range(wl.H):
+            ref = gu.oracle_lists(wl, int(classes[b, h]), block, permute)
+            assert small.lists(b, h) == [ref[a] for a in range(small.sched.nQ)], (seed, b, h, block)
     if seed % 4 == 0:
         Od, lsed = run.dense()
         Or, lr = orc.masked_attention(run.q_bits[0, 1], run.k_bits[0, 1], run.v_bits[0, 1], orc.DENSE, g, pp)

@@ -555,7 +555,10 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         }
         const float m_use = m_run == -INFINITY ? 0.f : m_run;
         const float2 sc2 = make_float2(sc, sc), mneg = make_float2(-m_use, -m_use);
-        float2 la = make_float2(0.f, 0.f), lb = make_float2(0.f, 0.f);
+        // several partial sums, so that the chain of dependent additions left after the last exponential is
+        // short (the sum of the rounded weights gates the P store)
+        float2 la[2], lb[4];
+        la[0] = la[1] = lb[0] = lb[1] = lb[2] = lb[3] = make_float2(0.f, 0.f);
 #pragma unroll
         for (int c = 0; c < 128; c += 4) {
           float2 e0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, mneg);
@@ -564,10 +567,12 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           e1.x = ex2(e1.x); e1.y = ex2(e1.y);
           pk[c / 2] = pack_bf16(e0.x, e0.y);
           pk[c / 2 + 1] = pack_bf16(e1.x, e1.y);
-          la = __fadd2_rn(la, __fadd2_rn(e0, e1));
-          lb = __fadd2_rn(lb, __fadd2_rn(unpack_bf16(pk[c / 2]), unpack_bf16(pk[c / 2 + 1])));
+          la[(c >> 2) & 1] = __fadd2_rn(la[(c >> 2) & 1], __fadd2_rn(e0, e1));
+          lb[(c >> 2) & 3] = __fadd2_rn(lb[(c >> 2) & 3], __fadd2_rn(unpack_bf16(pk[c / 2]), unpack_bf16(pk[c / 2 + 1])));
         }
-        const float l_tile = lb.x + lb.y, l_tile_exact = la.x + la.y;
+        la[0] = __fadd2_rn(la[0], la[1]);
+        lb[0] = __fadd2_rn(__fadd2_rn(lb[0], lb[1]), __fadd2_rn(lb[2], lb[3]));
+        const float l_tile = lb[0].x + lb[0].y, l_tile_exact = la[0].x + la[0].y;
         if (pass == 1) { l_run += l_tile; l_exact += l_tile_exact; break; }
         const bool bad = !(l_tile <= kSumLimit) || m_run == -INFINITY;
         if (!__any_sync(0xffffffffu, bad)) { l_run += l_tile; l_exact += l_tile_exact; break; }

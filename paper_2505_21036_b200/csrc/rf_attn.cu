@@ -334,18 +334,22 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
       const uint32_t v_lo = ((base + C::V0) >> 4) | LO_VMAJOR;
       auto issue_s = [&](int j, int ks) {
         const uint32_t a0 = q_lo + j * (C::TILE >> 4), b0 = k_lo + ks * (C::TILE >> 4);
+        // the accumulate flag is a compile-time constant: the issuing thread blocks on every MMA, so each
+        // instruction between two of them is idle tensor time
+        const uint32_t t_d = tmem_base + (j ? C::S_COL1 : C::S_COL0);
+        mma_ss_c<false>(t_d, desc(a0), desc(b0), IDESC_S);
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          mma_ss(tmem_base + (j ? C::S_COL1 : C::S_COL0), desc(a0 + (C::koff(k) >> 4)), desc(b0 + (C::koff(k) >> 4)),
-                 IDESC_S, k > 0);
+        for (int k = 1; k < D / 16; ++k)
+          mma_ss_c<true>(t_d, desc(a0 + (C::koff(k) >> 4)), desc(b0 + (C::koff(k) >> 4)), IDESC_S);
         tc_commit(bar(C::B_SF + j));
       };
       auto issue_pv = [&](int j, int vs, bool first) {
         const uint32_t b0 = v_lo + vs * (C::TILE >> 4);
         const uint32_t t_p = tmem_base + (j ? C::P_COL1 : C::P_COL0), t_o = tmem_base + (j ? C::O_COL1 : C::O_COL0);
+        mma_ts(t_o, t_p, desc(b0), IDESC_PV, !first);
 #pragma unroll
-        for (int k = 0; k < BN / 16; ++k)
-          mma_ts(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV, (!first) || k > 0);
+        for (int k = 1; k < BN / 16; ++k)
+          mma_ts_c<true>(t_o, t_p + k * 8, desc(b0 + k * (2048 >> 4)), IDESC_PV);
         tc_commit(bar(C::B_OF + j));
       };
       Merge mg;

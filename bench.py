@@ -247,7 +247,7 @@ def run_cuda(args, wl):
 
     def e2e_step():
         staged(qh, kh, vh, oh)
-    e2e_n = max(2, min(args.steps, 3))
+    e2e_n = max(2, min(args.steps, 10))
     e2e_step()
     barrier()
     a, b = ev(), ev()
@@ -291,7 +291,8 @@ def run_cuda(args, wl):
             "clocks": clocks,
             "e2e": {"value": dist_util.replica_throughput(dflops, e2e_ms, world) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": staged.h2d_bytes, "d2h_bytes_per_step": staged.d2h_bytes,
-                    "head_groups": groups, "equals_resident_output": e2e_same},
+                    "head_groups": groups, "equals_resident_output": e2e_same, "steps": e2e_n,
+                    "overlap": "head groups inside a step; copy-in of the next step under the kernels of this one"},
             "gpu_launches": args.steps * 5,   # rf_arm_kernel, rf_arm_decide_kernel, rf_build_tiles_kernel, rf_gather_kernel, rf_attn_kernel
             "breakdown_ms": {"arm": arm_ms, "block_mask": mask_ms, "sparse_attn_call": sparse_ms, "reorder": reorder_ms,
                              "attn_kernel": attn_kernel_ms, "dense_attn_call": dense_ms},

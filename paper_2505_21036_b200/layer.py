@@ -118,21 +118,25 @@ class HostStagedAttention:
         self.head_class = torch.zeros((groups, self.hg), dtype=torch.int32, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.s_in, self.s_run, self.s_out = (torch.cuda.Stream(device=device) for _ in range(3))
+        self._run_done, self._out_done = [], []      # per group, from the previous call
         self.h2d_bytes = 3 * heads * self.N * shape.D * 2
         self.d2h_bytes = heads * self.N * shape.D * 2
 
     def __call__(self, qh, kh, vh, oh):
-        """qh, kh, vh, oh: pinned host bf16 tensors of [B, H, N, D].  Returns when the work is enqueued; the
-        current stream waits for the output copy."""
+        """qh, kh, vh, oh: pinned host bf16 tensors of [B, H, N, D]; the inputs must be complete in host memory
+        when the call is made.  Returns when the work is enqueued; the current stream waits for the output copy.
+        Calls made back to back overlap: a group's staging buffers are refilled for the next call as soon as
+        this call's kernels are done with them, while later groups still compute."""
         import torch
         cur = torch.cuda.current_stream()
         hq, hk, hv, ho = (t.view(self.groups, self.hg, self.N, self.shape.D) for t in (qh, kh, vh, oh))
         dq, dk, dv, do = (t.view(self.groups, self.hg, self.N, self.shape.D) for t in (self.q, self.k, self.v, self.o))
-        for s in (self.s_in, self.s_run, self.s_out):
-            s.wait_stream(cur)
-        landed = []
+        prev_run, prev_out = self._run_done, self._out_done
+        landed, run_done, out_done = [], [], []
         with torch.cuda.stream(self.s_in):
             for g in range(self.groups):
+                if prev_run:
+                    self.s_in.wait_event(prev_run[g])      # the previous call's kernels have read this group's inputs
                 dq[g].copy_(hq[g], non_blocking=True)
                 dk[g].copy_(hk[g], non_blocking=True)
                 dv[g].copy_(hv[g], non_blocking=True)
@@ -142,6 +146,8 @@ class HostStagedAttention:
         for g in range(self.groups):
             with torch.cuda.stream(self.s_run):
                 self.s_run.wait_event(landed[g])
+                if prev_out:
+                    self.s_run.wait_event(prev_out[g])     # the previous call's output of this group has left
                 hc = self.head_class[g:g + 1]
                 api.rf_arm_classify(self.gshape, self.params, dq[g], dk[g], hc, None, self.ws)
                 api.rf_build_block_mask(self.gshape, self.params, hc, self.sched, self.status)
@@ -149,8 +155,12 @@ class HostStagedAttention:
                                        self.status)
                 done = torch.cuda.Event()
                 done.record()
+                run_done.append(done)
             with torch.cuda.stream(self.s_out):
                 self.s_out.wait_event(done)
                 ho[g].copy_(do[g], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record()
+                out_done.append(ev)
+        self._run_done, self._out_done = run_done, out_done
         cur.wait_stream(self.s_out)
-        cur.wait_stream(self.s_run)

@@ -88,3 +88,28 @@ def test_host_staged_call_equals_the_resident_pipeline(groups):
     assert torch.equal(oh.view(torch.int16), o.cpu().view(torch.int16))
     with pytest.raises(ValueError):
         HostStagedAttention(api.shape_of(wl), api.params_of(wl), "cuda", groups=3)
+
+
+@pytest.mark.gpu
+def test_host_staged_calls_back_to_back_with_different_inputs():
+    """Consecutive calls overlap (the next call's copy-in runs under this call's kernels): each call's output must
+    still belong to its own inputs."""
+    wl, eager = make_layer("cuda", dense_fraction=0.0)
+    from paper_2505_21036_b200.layer import HostStagedAttention
+    staged = HostStagedAttention(api.shape_of(wl), api.params_of(wl), "cuda", groups=2)
+    base = [torch.from_numpy(x.view(np.int16)).view(torch.bfloat16) for x in synth.make_qkv(wl)]
+    sets = []
+    for shift in range(4):                      # heads rotated: other classes, other schedules, other outputs
+        sets.append([torch.roll(t, shift, dims=1).contiguous().pin_memory() for t in base])
+    outs = [torch.full(base[0].shape, float("nan"), dtype=torch.bfloat16).pin_memory() for _ in sets]
+    for inp, out in zip(sets, outs):            # no synchronisation in between
+        staged(*inp, out)
+    torch.cuda.synchronize()
+    assert int(staged.status.item()) == 0
+    for inp, out in zip(sets, outs):
+        q, k, v = (t.cuda() for t in inp)
+        o = torch.empty_like(q)
+        eager(q, k, v, o, None, step=0, num_steps=1)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), o.cpu().view(torch.int16))
+    assert not torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))

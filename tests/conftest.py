@@ -20,3 +20,11 @@ def pytest_collection_modifyitems(config, items):
 @pytest.fixture(scope="session")
 def repo_root():
     return ROOT
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_library():
+    """The shared library is built in-tree once per session if it is missing or older than its sources
+    (nvcc cross-compiles without a GPU); a failing build fails the tests that need it, loudly."""
+    from paper_2505_21036_b200 import build
+    return build.build()

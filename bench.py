@@ -54,11 +54,13 @@ class ClockSampler:
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
+    def __init__(self, gpu_id: str):
+        """gpu_id: what `nvidia-smi -i` takes.  Pass the device's UUID ("GPU-..."): the CUDA ordinal is not the
+        nvidia-smi index when CUDA_VISIBLE_DEVICES reorders or hides GPUs of a shared machine."""
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.proc = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.QUERY}",
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.QUERY}",
                                           "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
@@ -182,7 +184,7 @@ def run_cuda(args, wl):
     def step(events=None):
         if events:
             events[0].record()
-        api.rf_arm_classify(shape, params, q, k, head_class, None, ws)   # classes only, as Algorithm 1 needs
+        api.rf_arm_classify(shape, params, q, k, head_class, None, ws, status)   # classes only, as Algorithm 1 needs
         if events:
             events[1].record()
         api.rf_build_block_mask(shape, params, head_class, sched, status)
@@ -207,7 +209,11 @@ def run_cuda(args, wl):
     if int(status.item()) != 0:
         raise SystemExit(f"bench.py: device status {int(status.item())}")
 
-    sampler = ClockSampler(local) if rank == 0 else None
+    try:
+        gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:                      # no uuid attribute: fall back to the ordinal and say so in the line
+        gpu_uuid = None
+    sampler = ClockSampler(gpu_uuid if gpu_uuid else str(local)) if rank == 0 else None
     per = [[ev() for _ in range(5)] for _ in range(args.steps)]
     t_begin, t_end = ev(), ev()
     barrier()
@@ -263,7 +269,7 @@ def run_cuda(args, wl):
     torch.cuda.synchronize()
     e2e_same = bool(torch.equal(oh.view(torch.int16), o.cpu().view(torch.int16)))   # same bits as the resident path
 
-    api.rf_arm_classify(shape, params, q, k, head_class, recall, ws)       # untimed: recalls for the report
+    api.rf_arm_classify(shape, params, q, k, head_class, recall, ws, status)       # untimed: recalls for the report
     torch.cuda.synchronize()
     rec = recall.cpu().numpy().reshape(-1, 3)
     cls = head_class.cpu().numpy().reshape(-1)
@@ -288,7 +294,7 @@ def run_cuda(args, wl):
                        "frame_window": wl.frame_window, "spatial_window": wl.spatial_window,
                        "textural_stride": wl.textural_stride, "sample_stride": wl.sample_stride,
                        "l2": f"inputs ({3 * wl.B * wl.H * wl.N * wl.D * 2 / 1e9:.2f} GB of Q/K/V) exceed the 126 MB L2; no flush", "parallelism": f"replicas x{world}"},
-            "clocks": clocks,
+            "clocks": dict(clocks or {}, gpu=gpu_uuid if gpu_uuid else f"ordinal {local}"),
             "e2e": {"value": dist_util.replica_throughput(dflops, e2e_ms, world) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": staged.h2d_bytes, "d2h_bytes_per_step": staged.d2h_bytes,
                     "head_groups": groups, "equals_resident_output": e2e_same, "steps": e2e_n,
@@ -340,6 +346,29 @@ def run_cuda(args, wl):
     dist_util.shutdown()
 
 
+def run_stub(args, wl):
+    """The rank bookkeeping of the CUDA arm without a GPU (used by the CPU tests of the N > 1 path): gloo
+    backend, a step that only sleeps, the same barrier / max-over-ranks / replica-throughput arithmetic and
+    the same "rank 0 prints one line" rule.  Nothing of the method runs here and no number it prints is a
+    measurement."""
+    from paper_2505_21036_b200 import dist_util
+    rank, world, _ = dist_util.env_rank()
+    dist_util.init("gloo")
+    dist_util.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.01 * (1 + rank))
+    ms = 1e3 * (time.perf_counter() - t0) / args.steps
+    dist_util.barrier()
+    (ms_max,) = dist_util.max_over_ranks([ms])
+    if rank == 0:
+        print(json.dumps({"impl": "stub", "metric": METRIC, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": ms_max, "scaling": "weak",
+                          "value": dist_util.replica_throughput(dense_flops(wl), ms_max, world) / 1e12,
+                          "config": {"workload": wl.name, "parallelism": f"replicas x{world}"}}))
+    dist_util.shutdown()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -351,10 +380,21 @@ def main():
     ap.add_argument("--e2e-groups", type=int, default=0, help="head groups of the host-staged leg (0: automatic)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
     ap.add_argument("--no-dense", dest="dense", action="store_false", help="skip the dense-baseline timing")
+    ap.add_argument("--stub", action="store_true", help=argparse.SUPPRESS)   # CPU test of the N > 1 bookkeeping
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
-        run_reference(args, wl)
+        run_reference(args, wl)                    # rank 0 alone works; started bare, this process is rank 0
+        return
+    from paper_2505_21036_b200 import dist_util
+    if args.gpus > 1 and not dist_util.launched_by_torchrun():
+        # started bare: become the launcher of N independent replicas, one process per GPU
+        sys.exit(dist_util.spawn_replicas([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus))
+    _, world, _ = dist_util.env_rank()
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}")
+    if args.stub:
+        run_stub(args, wl)
     else:
         run_cuda(args, wl)
 

@@ -19,7 +19,13 @@
  *     no state between calls apart from per-device kernel attributes set on first use.
  *   - Host-detectable errors return a code before anything is launched.  Device-detected ones
  *     (a bounded wait that ran out, a head class outside 0..3) are written to *dev_status
- *     (device int32, may be NULL; never reset by the library) and the kernels still terminate.
+ *     (device int32, may be NULL; never reset by the library; the first error stays) and the kernels
+ *     still terminate.  Every entry point that launches a kernel with such a wait takes a dev_status.
+ *     If a wait runs out inside ARM, head_class (and head_window) are written as -1 for every head, so
+ *     that rf_build_block_mask and rf_sparse_attn_fwd, given those classes, report RF_ERR_INVALID_ARG
+ *     through their own dev_status even when ARM itself was given none.
+ *   - frame_window >= T, spatial_window >= frame_h*frame_w and textural_stride >= max(frame_h, frame_w)
+ *     are accepted and mean what the extent itself means (all frames, all positions, the diagonal y == x).
  *   - Supported: D in {64, 96, 128}; block_m = block_n = 128 for the attention entry points;
  *     rf_build_block_mask alone accepts any power-of-two blocks >= 16.
  */
@@ -106,9 +112,12 @@ size_t rf_workspace_bytes(const rf_shape *shape, const rf_params *params);
  *   head_class  device int32 [B,H], written
  *   recall      device float [B,H,3] = (R_temporal, R_spatial, R_textural), written; may be NULL
  *   ws          device workspace of at least rf_workspace_bytes(), 256-byte aligned
+ *   dev_status  device int32 or NULL: RF_ERR_TIMEOUT if a wait inside the score kernel ran out (head_class
+ *               is then -1 for every head and recall is left unwritten)
  */
 rf_status rf_arm_classify(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
-                          int32_t *head_class, float *recall, void *ws, size_t ws_bytes, void *cuda_stream);
+                          int32_t *head_class, float *recall, void *ws, size_t ws_bytes, int32_t *dev_status,
+                          void *cuda_stream);
 
 /*
  * Block mask / tile schedule of the pattern masks of Sec. 3.2 (Eq. 3-5), per head, from device-resident
@@ -164,6 +173,17 @@ rf_status rf_sparse_attn_reordered(const rf_shape *shape, const rf_params *param
  */
 rf_status rf_selftest_wait_timeout(int32_t *dev_status, int32_t limit_ms, int32_t *waits_returned, void *cuda_stream);
 
+/*
+ * Self-test of ARM's failure reporting (no counterpart in the paper).  Runs rf_arm_classify's launch sequence
+ * with the score kernel left out and its failure flag set instead, exactly as a wait that ran out inside that
+ * kernel leaves it.  Nothing waits and nothing stalls.  Afterwards head_class is -1 for every head and
+ * *dev_status is RF_ERR_TIMEOUT if it was 0 before; rf_build_block_mask / rf_sparse_attn_fwd given those
+ * classes report RF_ERR_INVALID_ARG through their dev_status.  Arguments as for rf_arm_classify.
+ */
+rf_status rf_selftest_arm_abandoned(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
+                                    int32_t *head_class, void *ws, size_t ws_bytes, int32_t *dev_status,
+                                    void *cuda_stream);
+
 /* Full 3D attention (Eq. 1-2, all-zero mask): the same kernel walking every tile.  ws may be NULL. */
 rf_status rf_dense_attn_fwd(const rf_shape *shape, const void *q, const void *k, const void *v, void *o,
                             float *lse, void *ws, size_t ws_bytes, int32_t *dev_status, void *cuda_stream);
@@ -177,13 +197,15 @@ rf_status rf_dense_attn_fwd(const rf_shape *shape, const void *q, const void *k,
  *   bandwidths   host float [n_bandwidths], ascending, each in (0, 1]
  *   head_window  device int32 [B,H], written: w_s of a Temporal head, w_f of a Spatial head, -1 for Textural
  *   recall       device float [B,H,2,n_bandwidths] = (Temporal, Spatial) x candidate, written; may be NULL
+ *   dev_status   as for rf_arm_classify (head_class and head_window are -1 after a wait that ran out)
  * rf_build_block_mask_plus / rf_sparse_attn_fwd_plus are rf_build_block_mask / rf_sparse_attn_fwd with those
  * per-head windows in place of params->frame_window / spatial_window (head_window == NULL: identical to them).
  */
 #define RF_MAX_BANDWIDTHS 4
 rf_status rf_arm_classify_plus(const rf_shape *shape, const rf_params *params, const float *bandwidths,
                                int32_t n_bandwidths, const void *q, const void *k, int32_t *head_class,
-                               int32_t *head_window, float *recall, void *ws, size_t ws_bytes, void *cuda_stream);
+                               int32_t *head_window, float *recall, void *ws, size_t ws_bytes, int32_t *dev_status,
+                               void *cuda_stream);
 rf_status rf_build_block_mask_plus(const rf_shape *shape, const rf_params *params, const int32_t *head_class,
                                    const int32_t *head_window, rf_schedule *out, int32_t *dev_status, void *cuda_stream);
 rf_status rf_sparse_attn_fwd_plus(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
@@ -202,20 +224,22 @@ rf_status rf_sparse_attn_fwd_plus(const rf_shape *shape, const rf_params *params
  * a fixed array inside the library's device image: RF_ARM_STATIC_SCRATCH_FLOATS floats (4 MiB) that
  * every GPU which loads the library holds until the process exits.
  *
- *   - Limit: 2 * B * H * 3 * roundup64(max(frame_h*frame_w, ceil(T*frame_h*frame_w / sample_stride)))
- *     floats must fit (the HunyuanVideo-720p layer needs 525 312).  Larger problems are rejected
+ *   - Limit: 2 * B * H * 3 * roundup64(max(frame_h*frame_w, ceil(T*frame_h*frame_w / sample_stride))) + 64
+ *     floats must fit (the HunyuanVideo-720p layer needs 525 376).  Larger problems are rejected
  *     with RF_ERR_STATIC_SCRATCH_TOO_SMALL before anything is launched.
  *   - Allocates nothing: no cudaMalloc / cudaFree, no allocating library call.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  *     that device current).  Make that first call outside any stream capture.
- *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it has to
- *     start at zero (every element that is read was written earlier in the same call), but two calls
- *     that overlap on the GPU - different streams, or different host threads - race on it.  Serialise
- *     them, or use rf_arm_classify with separate workspaces.
+ *   - All calls share the one array and it keeps the previous call's contents.  The one word of it that
+ *     has to start at zero (the flag that records a wait that ran out) is cleared by every call on its
+ *     stream before its kernels run; every other element that is read was written earlier in the same
+ *     call.  But two calls that overlap on the GPU - different streams, or different host threads -
+ *     race on the array.  Serialise them, or use rf_arm_classify with separate workspaces.
+ *   - dev_status: as for rf_arm_classify.
  */
 #define RF_ARM_STATIC_SCRATCH_FLOATS (1u << 20)
 rf_status rf_arm_classify_noalloc(const rf_shape *shape, const rf_params *params, const void *q, const void *k,
-                                  int32_t *head_class, float *recall, void *cuda_stream);
+                                  int32_t *head_class, float *recall, int32_t *dev_status, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -20,7 +20,7 @@ _lib = None
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
            "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
            "rf_arm_classify_noalloc", "rf_selftest_wait_timeout", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus",
-           "rf_sparse_attn_reordered"]
+           "rf_sparse_attn_reordered", "rf_selftest_arm_abandoned"]
 
 
 class rf_shape(C.Structure):
@@ -63,21 +63,23 @@ def load():
     lib.rf_workspace_bytes.restype = Z
     lib.rf_workspace_bytes.argtypes = [P(rf_shape), P(rf_params)]
     lib.rf_arm_classify.restype = I
-    lib.rf_arm_classify.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, Z, V]
+    lib.rf_arm_classify.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, Z, V, V]
     lib.rf_arm_classify_noalloc.restype = I
-    lib.rf_arm_classify_noalloc.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V]
+    lib.rf_arm_classify_noalloc.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, V]
     lib.rf_build_block_mask.restype = I
     lib.rf_build_block_mask.argtypes = [P(rf_shape), P(rf_params), V, P(rf_schedule), V, V]
     lib.rf_sparse_attn_fwd.restype = I
     lib.rf_sparse_attn_fwd.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
     lib.rf_arm_classify_plus.restype = I
-    lib.rf_arm_classify_plus.argtypes = [P(rf_shape), P(rf_params), P(C.c_float), C.c_int32, V, V, V, V, V, V, Z, V]
+    lib.rf_arm_classify_plus.argtypes = [P(rf_shape), P(rf_params), P(C.c_float), C.c_int32, V, V, V, V, V, V, Z, V, V]
     lib.rf_build_block_mask_plus.restype = I
     lib.rf_build_block_mask_plus.argtypes = [P(rf_shape), P(rf_params), V, V, P(rf_schedule), V, V]
     lib.rf_sparse_attn_fwd_plus.restype = I
     lib.rf_sparse_attn_fwd_plus.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, V, P(rf_schedule), V, V, V, Z, V, V]
     lib.rf_sparse_attn_reordered.restype = I
     lib.rf_sparse_attn_reordered.argtypes = lib.rf_sparse_attn_fwd_plus.argtypes
+    lib.rf_selftest_arm_abandoned.restype = I
+    lib.rf_selftest_arm_abandoned.argtypes = [P(rf_shape), P(rf_params), V, V, V, V, Z, V, V]
     lib.rf_selftest_wait_timeout.restype = I
     lib.rf_selftest_wait_timeout.argtypes = [V, C.c_int32, V, V]
     lib.rf_reorder_tokens.restype = I
@@ -158,18 +160,19 @@ def alloc_workspace(shape: rf_shape, params: rf_params, device):
     return torch.empty(rf_workspace_bytes(shape, params), dtype=torch.uint8, device=device)
 
 
-def rf_arm_classify(shape, params, q, k, head_class, recall, ws):
+def rf_arm_classify(shape, params, q, k, head_class, recall, ws, dev_status=None):
     _check(load().rf_arm_classify(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(), head_class.data_ptr(),
-                                  _ptr(recall), ws.data_ptr(), ws.numel(), _stream()), "rf_arm_classify")
+                                  _ptr(recall), ws.data_ptr(), ws.numel(), _ptr(dev_status), _stream()), "rf_arm_classify")
 
 
-def rf_arm_classify_noalloc(shape, params, q, k, head_class, recall):
+def rf_arm_classify_noalloc(shape, params, q, k, head_class, recall, dev_status=None):
     """rf_arm_classify without a workspace: for callers that may not allocate device memory (a frozen
     serving pool, a plug-in that must not re-enter the framework allocator).  The scratch is a fixed
     4 MiB array inside the library; problems that need more raise RainFusionError.  Calls that overlap
     on the GPU share that array and race; run them one after the other."""
     _check(load().rf_arm_classify_noalloc(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(),
-                                          head_class.data_ptr(), _ptr(recall), _stream()), "rf_arm_classify_noalloc")
+                                          head_class.data_ptr(), _ptr(recall), _ptr(dev_status), _stream()),
+           "rf_arm_classify_noalloc")
 
 
 def rf_build_block_mask(shape, params, head_class, sched: Schedule, dev_status=None):
@@ -183,11 +186,11 @@ def rf_sparse_attn_fwd(shape, params, q, k, v, head_class, sched: Schedule, o, l
                                      ws.numel(), _ptr(dev_status), _stream()), "rf_sparse_attn_fwd")
 
 
-def rf_arm_classify_plus(shape, params, bandwidths, q, k, head_class, head_window, recall, ws):
+def rf_arm_classify_plus(shape, params, bandwidths, q, k, head_class, head_window, recall, ws, dev_status=None):
     arr = (C.c_float * len(bandwidths))(*bandwidths)
     _check(load().rf_arm_classify_plus(C.byref(shape), C.byref(params), arr, len(bandwidths), q.data_ptr(), k.data_ptr(),
                                        head_class.data_ptr(), head_window.data_ptr(), _ptr(recall), ws.data_ptr(),
-                                       ws.numel(), _stream()), "rf_arm_classify_plus")
+                                       ws.numel(), _ptr(dev_status), _stream()), "rf_arm_classify_plus")
 
 
 def rf_build_block_mask_plus(shape, params, head_class, head_window, sched: Schedule, dev_status=None):
@@ -212,6 +215,12 @@ def rf_sparse_attn_reordered(shape, params, q, k, v, head_class, head_window, sc
 def rf_selftest_wait_timeout(dev_status, limit_ms, waits_returned):
     _check(load().rf_selftest_wait_timeout(dev_status.data_ptr(), limit_ms, waits_returned.data_ptr(), _stream()),
            "rf_selftest_wait_timeout")
+
+
+def rf_selftest_arm_abandoned(shape, params, q, k, head_class, ws, dev_status):
+    _check(load().rf_selftest_arm_abandoned(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(),
+                                            head_class.data_ptr(), ws.data_ptr(), ws.numel(), _ptr(dev_status), _stream()),
+           "rf_selftest_arm_abandoned")
 
 
 def rf_reorder_tokens(shape, params, q, k, v, head_class, ws):

@@ -48,7 +48,13 @@ RfGeom make_geom(const rf_shape* s, int wf, int ws, int tau, int bm, int bn, int
   g.B = s->B; g.H = s->H; g.D = s->D;
   g.T = s->T; g.Hf = s->frame_h; g.Wf = s->frame_w; g.S = s->frame_h * s->frame_w;
   g.Nv = g.T * g.S; g.L = s->L_text; g.N = g.Nv + g.L;
-  g.wf = wf; g.ws = ws; g.tau = tau;
+  // Windows past the extent and strides past the frame's longer side give the same masks as the extent itself
+  // (every frame / position within reach; y mod tau = y and x mod tau = x); clamping keeps the kernels' index
+  // arithmetic ((f + w_f + 1) * S, p + w_s, loops over tau) inside int range for any caller value.
+  g.wf = wf < g.T ? wf : g.T;
+  g.ws = ws < g.S ? ws : g.S;
+  g.tau = tau < (g.Hf > g.Wf ? g.Hf : g.Wf) ? tau : (g.Hf > g.Wf ? g.Hf : g.Wf);
+  tau = g.tau;
   g.nC = checkerboard_count(g.Hf, g.Wf, tau);
   g.LkvTex = g.T * g.nC + g.L;
   g.BM = bm; g.BN = bn;
@@ -209,7 +215,8 @@ size_t rf_workspace_bytes(const rf_shape* shape, const rf_params* params) {
 }
 
 rf_status rf_arm_classify(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
-                          int32_t* head_class, float* recall, void* ws, size_t ws_bytes, void* cuda_stream) {
+                          int32_t* head_class, float* recall, void* ws, size_t ws_bytes, int32_t* dev_status,
+                          void* cuda_stream) {
   rf_status st = check_shape(shape);
   if (st != RF_OK) return st;
   st = check_params(params);
@@ -222,13 +229,32 @@ rf_status rf_arm_classify(const rf_shape* shape, const rf_params* params, const 
   float* scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + 3 * tensor_bytes(g));
   cudaError_t e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, 1, &g.ws, &g.wf,
                                 static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), head_class,
-                                nullptr, recall, nullptr, scratch, static_cast<cudaStream_t>(cuda_stream));
+                                nullptr, recall, nullptr, scratch, dev_status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
+}
+
+rf_status rf_selftest_arm_abandoned(const rf_shape* shape, const rf_params* params, const void* q, const void* k,
+                                    int32_t* head_class, void* ws, size_t ws_bytes, int32_t* dev_status, void* cuda_stream) {
+  rf_status st = check_shape(shape);
+  if (st != RF_OK) return st;
+  st = check_params(params);
+  if (st != RF_OK) return st;
+  if (shape->D != 64 && shape->D != 96 && shape->D != 128) return RF_ERR_UNSUPPORTED;
+  if (q == nullptr || k == nullptr || head_class == nullptr || ws == nullptr) return RF_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return RF_ERR_INVALID_ARG;
+  if (ws_bytes < rf_workspace_bytes(shape, params)) return RF_ERR_WORKSPACE_TOO_SMALL;
+  const RfGeom g = make_geom(shape, params);
+  float* scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + 3 * tensor_bytes(g));
+  cudaError_t e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, 1, &g.ws, &g.wf,
+                                static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), head_class,
+                                nullptr, nullptr, nullptr, scratch, dev_status, static_cast<cudaStream_t>(cuda_stream), true);
   return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }
 
 rf_status rf_arm_classify_plus(const rf_shape* shape, const rf_params* params, const float* bandwidths,
                                int32_t n_bandwidths, const void* q, const void* k, int32_t* head_class,
-                               int32_t* head_window, float* recall, void* ws, size_t ws_bytes, void* cuda_stream) {
+                               int32_t* head_window, float* recall, void* ws, size_t ws_bytes, int32_t* dev_status,
+                               void* cuda_stream) {
   rf_status st = check_shape(shape);
   if (st != RF_OK) return st;
   st = check_params(params);
@@ -249,7 +275,8 @@ rf_status rf_arm_classify_plus(const rf_shape* shape, const rf_params* params, c
   float* scratch = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + 3 * tensor_bytes(g));
   cudaError_t e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, n_bandwidths, ws_list,
                                 wf_list, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
-                                head_class, head_window, nullptr, recall, scratch, static_cast<cudaStream_t>(cuda_stream));
+                                head_class, head_window, nullptr, recall, scratch, dev_status,
+                                static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }
 

@@ -18,6 +18,11 @@
 // need per-key attributes, computed cooperatively per tile.
 // Per-row recalls go to scratch; a second kernel averages them in a fixed order (deterministic) and
 // takes Algorithm 1's decision.  The n x n score matrix is never written.
+// A bounded wait that runs out is recorded in a flag word at the end of the scratch (cleared at the start of
+// every call); the decision kernel then writes class -1 for every head instead of a class computed from
+// unwritten rows, and passes the code on to the caller's status word.  The tile builder and the attention
+// kernel report a class outside 0..3 through their own status, so the failure cannot go unnoticed even by a
+// caller that gave ARM no status pointer.
 #include "rf_sm100.cuh"
 
 namespace {
@@ -25,7 +30,7 @@ namespace {
 using namespace sm100;
 
 constexpr int ARM_TILE = 128;
-constexpr int ARM_THREADS = 384;           // softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
+constexpr int ARM_THREADS = kWsThreads;    // softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
 constexpr int ARM_TMA_WARP = 8, ARM_MMA_WARP = 9;
 
 struct ArmMaps { CUtensorMap q[2], k[2]; };   // per sample: 0 = stride sample, 1 = first-frame sample
@@ -84,7 +89,7 @@ template <int D, int NB, bool TEX>
 __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_constant__ ArmMaps maps, const RfGeom g,
                                                                 const ArmSample sm0, const ArmSample sm1,
                                                                 const ArmWindows win, int n_pad, float scale_log2,
-                                                                int32_t* dev_status) {
+                                                                int32_t* arm_flag) {
   using C = ArmCfg<D>;
   constexpr uint32_t IDESC_S = idesc_bf16(128, 128, 0);
   extern __shared__ uint8_t smem_raw[];
@@ -126,10 +131,10 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const WaitCtx wc{abort_flag, dev_status};
+  const WaitCtx wc{abort_flag, arm_flag};
 
   if (warp >= 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    RF_SETMAXNREG_DEC();
     if (warp == ARM_TMA_WARP) {
       if (lane == 0) {
         mbar_expect_tx(bar(C::B_Q), 2 * C::TILE);
@@ -172,7 +177,7 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
       }
     }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    RF_SETMAXNREG_INC();
     const int j = warp >> 2;
     if (j == 0 || stream1) {
       const int m = (qt0 + j) * ARM_TILE + (tid & 127);          // sampled row of this thread
@@ -355,10 +360,21 @@ __global__ void __launch_bounds__(256) rf_arm_decide_kernel(int nb, int nb_user,
                                                              const float* __restrict__ rows_glb,
                                                              int32_t* __restrict__ head_class,
                                                              int32_t* __restrict__ head_window, float* __restrict__ recall,
-                                                             float* __restrict__ recall_plus) {
+                                                             float* __restrict__ recall_plus,
+                                                             const int32_t* __restrict__ arm_flag, int32_t* dev_status) {
   __shared__ double red[2 * ARM_MAX_NB + 1][256];
   const int bh = blockIdx.x, tid = threadIdx.x;
   const int nm = 2 * nb + 1;
+  const int failed = *arm_flag;
+  if (failed != 0) {
+    // the score kernel gave up a wait: its rows are incomplete, no class may come out of them
+    if (tid == 0) {
+      rf_report(dev_status, failed);
+      head_class[bh] = -1;
+      if (head_window != nullptr) head_window[bh] = -1;
+    }
+    return;
+  }
   const float* gl = rows_glb + (size_t)bh * nm * n_pad;
   const float* lo = rows_loc + (size_t)bh * nm * n_pad;
   const bool local_t = sample_mode == RF_SAMPLE_ALG1;
@@ -409,30 +425,34 @@ __global__ void __launch_bounds__(256) rf_arm_decide_kernel(int nb, int nb_user,
   }
 }
 
+// Self-test only: stands in for a score kernel whose wait ran out.
+__global__ void rf_arm_set_flag_kernel(int32_t* arm_flag, int code) { *arm_flag = code; }
+
 template <int D, int NB, bool TEX>
 cudaError_t launch_arm_t(const ArmMaps& maps, const RfGeom& g, const ArmSample& s0, const ArmSample& s1,
-                         const ArmWindows& win, int n_pad, int32_t* dev_status, cudaStream_t st) {
+                         const ArmWindows& win, int n_pad, int32_t* arm_flag, cudaStream_t st) {
   static bool configured[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (!rf_regs_ok(rf_arm_kernel<D, NB, TEX>)) return cudaErrorLaunchOutOfResources;   // setmaxnreg.inc could never be granted
     e = cudaFuncSetAttribute(rf_arm_kernel<D, NB, TEX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ArmCfg<D>::ALLOC);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   dim3 grid(s0.pairs + s1.pairs, g.B * g.H);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
-  rf_arm_kernel<D, NB, TEX><<<grid, ARM_THREADS, ArmCfg<D>::ALLOC, st>>>(maps, g, s0, s1, win, n_pad, scale_log2, dev_status);
+  rf_arm_kernel<D, NB, TEX><<<grid, ARM_THREADS, ArmCfg<D>::ALLOC, st>>>(maps, g, s0, s1, win, n_pad, scale_log2, arm_flag);
   return cudaGetLastError();
 }
 
 template <int D>
 cudaError_t launch_arm_n(bool plus, bool tex, const ArmMaps& maps, const RfGeom& g, const ArmSample& s0,
-                         const ArmSample& s1, const ArmWindows& win, int n_pad, cudaStream_t st) {
-  if (plus) return launch_arm_t<D, ARM_MAX_NB, false>(maps, g, s0, s1, win, n_pad, nullptr, st);
-  return tex ? launch_arm_t<D, 1, true>(maps, g, s0, s1, win, n_pad, nullptr, st)
-             : launch_arm_t<D, 1, false>(maps, g, s0, s1, win, n_pad, nullptr, st);
+                         const ArmSample& s1, const ArmWindows& win, int n_pad, int32_t* arm_flag, cudaStream_t st) {
+  if (plus) return launch_arm_t<D, ARM_MAX_NB, false>(maps, g, s0, s1, win, n_pad, arm_flag, st);
+  return tex ? launch_arm_t<D, 1, true>(maps, g, s0, s1, win, n_pad, arm_flag, st)
+             : launch_arm_t<D, 1, false>(maps, g, s0, s1, win, n_pad, arm_flag, st);
 }
 
 int arm_n_pad(const RfGeom& g, int omega) {
@@ -443,13 +463,15 @@ int arm_n_pad(const RfGeom& g, int omega) {
 
 }  // namespace
 
+// Per-row recalls of both samples, then RF_ARM_FLAG_FLOATS floats whose first word is the call's failure flag.
 size_t rf_arm_scratch_floats(const RfGeom& g, int omega, int nb) {
-  return (size_t)2 * g.B * g.H * (2 * nb + 1) * arm_n_pad(g, omega);
+  return (size_t)2 * g.B * g.H * (2 * nb + 1) * arm_n_pad(g, omega) + RF_ARM_FLAG_FLOATS;
 }
 
 cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, int nb, const int* ws_list,
                           const int* wf_list, const __nv_bfloat16* q, const __nv_bfloat16* k, int32_t* head_class,
-                          int32_t* head_window, float* recall, float* recall_plus, float* row_scratch, cudaStream_t st) {
+                          int32_t* head_window, float* recall, float* recall_plus, float* row_scratch, int32_t* dev_status,
+                          cudaStream_t st, bool selftest_abandon) {
   const bool plus = head_window != nullptr;
   const int NB = plus ? ARM_MAX_NB : 1;           // windows the kernel evaluates (candidate list padded by repetition)
   if (nb < 1 || nb > NB) return cudaErrorInvalidValue;
@@ -463,6 +485,7 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
   const int heads = g.B * g.H;
   float* rows_glb = row_scratch;
   float* rows_loc = row_scratch + (size_t)heads * (2 * NB + 1) * n_pad;
+  int32_t* arm_flag = reinterpret_cast<int32_t*>(row_scratch + (size_t)2 * heads * (2 * NB + 1) * n_pad);
   const bool alg1 = sample_mode == RF_SAMPLE_ALG1;
   const bool tex = !plus && recall != nullptr;   // the Textural recall is a diagnostic: Algorithm 1 does not use it
   const size_t row_bytes = (size_t)g.D * 2, head_bytes = (size_t)g.N * g.D * 2;
@@ -477,16 +500,21 @@ cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alp
   s0.want_t = alg1 ? 0 : 1; s0.want_s = 1; s0.out = rows_glb;
   s1.n = n_loc; s1.stride = 1; s1.pairs = alg1 ? rf_cdiv(rf_cdiv(n_loc, ARM_TILE), 2) : 0;
   s1.want_t = 1; s1.want_s = 0; s1.out = rows_loc;
-  cudaError_t e;
+  cudaError_t e = cudaMemsetAsync(arm_flag, 0, sizeof(int32_t), st);
+  if (e != cudaSuccess) return e;
+  if (selftest_abandon) {
+    rf_arm_set_flag_kernel<<<1, 1, 0, st>>>(arm_flag, RF_ERR_TIMEOUT);
+    e = cudaGetLastError();
+  } else
   switch (g.D) {
-    case 64: e = launch_arm_n<64>(plus, tex, maps, g, s0, s1, win, n_pad, st); break;
-    case 96: e = launch_arm_n<96>(plus, tex, maps, g, s0, s1, win, n_pad, st); break;
-    case 128: e = launch_arm_n<128>(plus, tex, maps, g, s0, s1, win, n_pad, st); break;
+    case 64: e = launch_arm_n<64>(plus, tex, maps, g, s0, s1, win, n_pad, arm_flag, st); break;
+    case 96: e = launch_arm_n<96>(plus, tex, maps, g, s0, s1, win, n_pad, arm_flag, st); break;
+    case 128: e = launch_arm_n<128>(plus, tex, maps, g, s0, s1, win, n_pad, arm_flag, st); break;
     default: e = cudaErrorInvalidValue;
   }
   if (e != cudaSuccess) return e;
   rf_arm_decide_kernel<<<heads, 256, 0, st>>>(NB, nb, n_loc, n_glb, n_pad, sample_mode, alpha, g.two_mask, win, tex ? 1 : 0, rows_loc,
-                                              rows_glb, head_class, head_window, recall, recall_plus);
+                                              rows_glb, head_class, head_window, recall, recall_plus, arm_flag, dev_status);
   return cudaGetLastError();
 }
 
@@ -515,7 +543,8 @@ float* static_scratch_ptr(int dev, cudaError_t* err) {
 }  // namespace
 
 extern "C" rf_status rf_arm_classify_noalloc(const rf_shape* shape, const rf_params* params, const void* q,
-                                             const void* k, int32_t* head_class, float* recall, void* cuda_stream) {
+                                             const void* k, int32_t* head_class, float* recall, int32_t* dev_status,
+                                             void* cuda_stream) {
   RfGeom g;
   rf_status st = rf_checked_geom(shape, params, &g);
   if (st != RF_OK) return st;
@@ -531,6 +560,6 @@ extern "C" rf_status rf_arm_classify_noalloc(const rf_shape* shape, const rf_par
   if (scratch == nullptr) return RF_ERR_CUDA;
   e = rf_launch_arm(g, params->sample_mode, params->sample_stride, params->alpha, 1, &g.ws, &g.wf,
                     static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), head_class, nullptr, recall,
-                    nullptr, scratch, static_cast<cudaStream_t>(cuda_stream));
+                    nullptr, scratch, dev_status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }

@@ -22,7 +22,7 @@ namespace {
 using namespace sm100;
 
 constexpr int BM = 128, BN = 128;
-constexpr int kThreads = 384;               // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
+constexpr int kThreads = kWsThreads;        // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
 constexpr int kTmaWarp = 8, kMmaWarp = 9;
 // Lazy rescaling of the running maximum.  A tile's weights are taken as 2^(score - running maximum) and accepted
 // while their row sum stays within kSumLimit; beyond it the row's maximum is raised.  bf16 P and the fp32 sums
@@ -232,8 +232,8 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   }
   if (a.head_window != nullptr) {   // dynamic bandwidth: this head's own window
     const int w = a.head_window[bh];
-    if (cls == RF_SPATIAL && w >= 0) g.wf = w;
-    if (cls == RF_TEMPORAL && w >= 0) g.ws = w;
+    if (cls == RF_SPATIAL && w >= 0) g.wf = min(w, g.T);     // past the extent: same mask, no overflow
+    if (cls == RF_TEMPORAL && w >= 0) g.ws = min(w, g.S);
   }
   const bool perm = cls == RF_TEMPORAL && g.permute;
   const bool tex = cls == RF_TEXTURAL;
@@ -281,7 +281,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   const WaitCtx wc{abort_flag, a.dev_status};
 
   if (warp >= 8) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+  RF_SETMAXNREG_DEC();
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -412,7 +412,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
     }
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    RF_SETMAXNREG_INC();
     // ------------------------------------------------------------ softmax + epilogue, one thread per query row
     const int j = warp >> 2;                       // stream
     const int row_in_tile = tid & 127;
@@ -660,6 +660,7 @@ rf_status launch(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st) 
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return RF_ERR_CUDA;
   if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (!rf_regs_ok(rf_attn_kernel<D>)) return RF_ERR_UNSUPPORTED;   // setmaxnreg.inc could never be granted
     if (cudaFuncSetAttribute(rf_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<D>::ALLOC) != cudaSuccess)
       return RF_ERR_CUDA;
     configured[dev] = true;

@@ -45,9 +45,15 @@ cudaError_t rf_launch_gather(const RfGeom& g, const int32_t* head_class, const _
 // nb candidate windows per pattern (ws_list for Temporal, wf_list for Spatial, ascending).  head_window == nullptr:
 // plain Algorithm 1 on the first candidate (recall: [B,H,3] or null).  Otherwise dynamic bandwidth: head_window
 // receives each head's chosen window, recall_plus ([B,H,2,nb] or null) the candidates' recalls.
+// dev_status (nullable) receives RF_ERR_TIMEOUT if a wait inside the score kernel ran out; head_class is then -1.
+// selftest_abandon: the score kernel is not launched; its failure flag is set instead, as if a wait had run out.
 cudaError_t rf_launch_arm(const RfGeom& g, int sample_mode, int omega, float alpha, int nb, const int* ws_list,
                           const int* wf_list, const __nv_bfloat16* q, const __nv_bfloat16* k, int32_t* head_class,
-                          int32_t* head_window, float* recall, float* recall_plus, float* row_scratch, cudaStream_t st);
+                          int32_t* head_window, float* recall, float* recall_plus, float* row_scratch, int32_t* dev_status,
+                          cudaStream_t st, bool selftest_abandon = false);
+// Floats of ARM scratch: the per-row recalls plus RF_ARM_FLAG_FLOATS at the end whose first word records a
+// wait that ran out inside the score kernel (cleared by every call before its kernels run).
+#define RF_ARM_FLAG_FLOATS 64
 size_t rf_arm_scratch_floats(const RfGeom& g, int omega, int nb);
 // Tensor map over bf16 rows: [heads][rows][D] with the given row and head strides in bytes (multiples of 16),
 // box = 64 columns x 128 rows, 128-byte swizzle, zero fill past `rows`.

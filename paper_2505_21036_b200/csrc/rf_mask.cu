@@ -77,8 +77,8 @@ __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int
   }
   if (head_window != nullptr) {   // dynamic bandwidth: this head's own window
     const int w = head_window[bh];
-    if (cls == RF_SPATIAL && w >= 0) g.wf = w;
-    if (cls == RF_TEMPORAL && w >= 0) g.ws = w;
+    if (cls == RF_SPATIAL && w >= 0) g.wf = min(w, g.T);     // past the extent: same mask, no overflow
+    if (cls == RF_TEMPORAL && w >= 0) g.ws = min(w, g.S);
   }
   const int Lkv = rf_kv_len(g, cls);
   const int nK = rf_cdiv(Lkv, g.BN);

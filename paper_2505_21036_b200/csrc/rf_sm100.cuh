@@ -63,6 +63,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
   return false;
 }
 
+// ---------------------------------------------------------------- register budget of warp-specialised CTAs
+// The attention and ARM kernels run 384 threads: two softmax warpgroups that raise their register count with
+// setmaxnreg.inc and one warpgroup (TMA, MMA, two filler warps) that lowers its own first.  setmaxnreg.inc waits,
+// without any bound, until the CTA's register pool can grant the request, and the pool is what the CTA got at
+// launch: registers per thread (as allocated by ptxas) x 384.  The split is therefore checked twice: at compile
+// time against the 64 K registers of an SM, and on the host before the first launch against the kernel's actual
+// allocation (rf_regs_ok), so that a different compiler allocation fails with an error instead of blocking.
+constexpr int kWsThreads = 384, kRegsLow = 72, kRegsHigh = 216;
+constexpr int kWsRegsNeeded = 128 * kRegsLow + 256 * kRegsHigh;
+static_assert(kWsRegsNeeded <= 65536, "setmaxnreg split exceeds the register file of an SM");
+static_assert(kRegsLow % 8 == 0 && kRegsHigh % 8 == 0 && kRegsHigh <= 255, "setmaxnreg takes multiples of 8 up to 255");
+#define RF_SETMAXNREG_DEC() asm volatile("setmaxnreg.dec.sync.aligned.u32 72;")
+#define RF_SETMAXNREG_INC() asm volatile("setmaxnreg.inc.sync.aligned.u32 216;")
+static_assert(kRegsLow == 72 && kRegsHigh == 216, "keep RF_SETMAXNREG_DEC / RF_SETMAXNREG_INC in step with kRegsLow / kRegsHigh");
+// Host: true when a kernel launched with kWsThreads threads owns enough registers for the split.
+template <typename K>
+inline bool rf_regs_ok(K kernel) {
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) return false;
+  return fa.numRegs * kWsThreads >= kWsRegsNeeded;
+}
+
 // ---------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

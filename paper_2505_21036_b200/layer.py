@@ -48,12 +48,13 @@ class RainFusionAttention:
     def _sparse(self, q, k, v, o, lse):
         s, p = self.shape, self.params
         if self.bandwidths:
-            api.rf_arm_classify_plus(s, p, self.bandwidths, q, k, self.head_class, self.head_window, None, self.ws)
+            api.rf_arm_classify_plus(s, p, self.bandwidths, q, k, self.head_class, self.head_window, None, self.ws,
+                                     self.status)
             api.rf_build_block_mask_plus(s, p, self.head_class, self.head_window, self.sched, self.status)
             api.rf_sparse_attn_fwd_plus(s, p, q, k, v, self.head_class, self.head_window, self.sched, o, lse, self.ws,
                                         self.status)
         else:
-            api.rf_arm_classify(s, p, q, k, self.head_class, None, self.ws)
+            api.rf_arm_classify(s, p, q, k, self.head_class, None, self.ws, self.status)
             api.rf_build_block_mask(s, p, self.head_class, self.sched, self.status)
             api.rf_sparse_attn_fwd(s, p, q, k, v, self.head_class, self.sched, o, lse, self.ws, self.status)
 
@@ -149,7 +150,7 @@ class HostStagedAttention:
                 if prev_out:
                     self.s_run.wait_event(prev_out[g])     # the previous call's output of this group has left
                 hc = self.head_class[g:g + 1]
-                api.rf_arm_classify(self.gshape, self.params, dq[g], dk[g], hc, None, self.ws)
+                api.rf_arm_classify(self.gshape, self.params, dq[g], dk[g], hc, None, self.ws, self.status)
                 api.rf_build_block_mask(self.gshape, self.params, hc, self.sched, self.status)
                 api.rf_sparse_attn_fwd(self.gshape, self.params, dq[g], dk[g], dv[g], hc, self.sched, do[g], None, self.ws,
                                        self.status)

@@ -71,14 +71,35 @@ def test_bad_shapes_and_pointers_are_rejected_before_cuda(lib):
     # null and misaligned pointers
     assert lib.rf_dense_attn_fwd(C.byref(s), None, 256, 256, 256, None, None, 0, None, None) == 1
     assert lib.rf_dense_attn_fwd(C.byref(s), 264, 256, 256, 256, None, None, 0, None, None) == 1
-    assert lib.rf_arm_classify(C.byref(s), C.byref(p), 256, 256, None, None, 256, 1 << 30, None) == 1
-    assert lib.rf_arm_classify(C.byref(s), C.byref(p), 256, 256, 256, None, 256, 16, None) == 3   # workspace too small
+    assert lib.rf_arm_classify(C.byref(s), C.byref(p), 256, 256, None, None, 256, 1 << 30, None, None) == 1
+    assert lib.rf_arm_classify(C.byref(s), C.byref(p), 256, 256, 256, None, 256, 16, None, None) == 3   # workspace too small
+    assert lib.rf_arm_classify(C.byref(s), C.byref(p), 256, 264, 256, None, 256, 1 << 30, 256, None) == 1  # misaligned k
+    assert lib.rf_selftest_arm_abandoned(C.byref(s), C.byref(p), 256, 256, None, 256, 1 << 30, None, None) == 1
+    assert lib.rf_selftest_arm_abandoned(C.byref(s), C.byref(p), 256, 256, 256, 256, 16, None, None) == 3
+    bw = (C.c_float * 2)(0.25, 0.5)
+    assert lib.rf_arm_classify_plus(C.byref(s), C.byref(p), bw, 2, 256, 256, 256, None, None, 256, 1 << 30, None, None) == 1
+    assert lib.rf_arm_classify_plus(C.byref(s), C.byref(p), bw, 2, 256, 256, 256, 256, None, 256, 16, 256, None) == 3
+    assert lib.rf_arm_classify_noalloc(C.byref(s), C.byref(p), 256, 256, None, None, 256, None) == 1
     sched = api.rf_schedule(256, 256, None, 256, 1, 1)                # wrong nQ / nKmax
     assert lib.rf_build_block_mask(C.byref(s), C.byref(p), 256, C.byref(sched), None, None) == 1
     p64 = api.params_of(wl, 64, 64)
     sched = api.rf_schedule(256, 256, None, 256, 5, 5)
     assert lib.rf_sparse_attn_fwd(C.byref(s), C.byref(p64), 256, 256, 256, 256, C.byref(sched), 256, None, 256,
                                   1 << 30, None, None) == 2            # attention needs 128 x 128 tiles
+
+
+def test_oversized_windows_and_strides_are_accepted_and_bounded(lib):
+    """A window past the extent or a checkerboard stride past the frame means what the extent means; the host
+    side must neither reject it nor loop over it (textural_stride = INT_MAX used to cost 2^31 iterations)."""
+    import time
+    wl = synth.WORKLOADS["tiny"]
+    s, p = api.shape_of(wl), api.params_of(wl)
+    base = api.rf_workspace_bytes(s, p)
+    p.frame_window = p.spatial_window = p.textural_stride = 2**31 - 1
+    t0 = time.time()
+    assert api.rf_workspace_bytes(s, p) == base
+    assert api.rf_schedule_dims(s, p) == (3, 3)
+    assert time.time() - t0 < 0.5
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -45,29 +45,34 @@ def check_lists(run, classes, tiles=None, heads=None):
         assert int(run.sched.kv_len[0, h]) == orc.kv_len(cls, gu.geom(wl), gu.pparams(wl))
 
 
-def check_rows(run, O, lse, classes, rows, heads):
+def check_rows(run, O, lse, classes, rows, heads, pp_of_head=None):
+    """pp_of_head: head -> PatternParams, where heads carry windows of their own (dynamic bandwidth)."""
     wl = run.wl
     worst = [0.0, 0.0, 0.0, 0.0]
     for h in heads:
+        pp = gu.pparams(wl) if pp_of_head is None else pp_of_head(h)
         Or, lr = orc.masked_attention(run.q_bits[0, h], run.k_bits[0, h], run.v_bits[0, h], int(classes[h]),
-                                      gu.geom(wl), gu.pparams(wl), rows=rows)
+                                      gu.geom(wl), pp, rows=rows)
         res = gu.check_attention(O[h][rows], lse[h][rows], Or, lr, f"{wl.name} head {h} class {classes[h]}")
         worst = [max(a, b) for a, b in zip(worst, res)]
     return worst
 
 
-def gpu_outputs(run, dense=False):
+def gpu_outputs(run, dense=False, plus=False):
     """O as float64 rows on demand would need the whole tensor on the host; keep bf16 there and widen per head."""
     wl = run.wl
-    o = torch.full((wl.B, wl.H, wl.N, wl.D), float("nan"), dtype=torch.bfloat16, device="cuda")
-    lse = torch.full((wl.B, wl.H, wl.N), float("nan"), dtype=torch.float32, device="cuda")
-    if dense:
-        api.rf_dense_attn_fwd(run.shape, run.q, run.k, run.v, o, lse, run.status)
+    if plus:
+        o, lse = run.sparse_plus(to_numpy=False)
     else:
-        api.rf_sparse_attn_fwd(run.shape, run.params, run.q, run.k, run.v, run.head_class, run.sched, o, lse, run.ws,
-                               run.status)
-    torch.cuda.synchronize()
-    assert int(run.status.item()) == 0
+        o, lse = run.outputs()                     # NaN-filled, between guard words
+        if dense:
+            api.rf_dense_attn_fwd(run.shape, run.q, run.k, run.v, o, lse, run.status)
+        else:
+            api.rf_sparse_attn_fwd(run.shape, run.params, run.q, run.k, run.v, run.head_class, run.sched, o, lse, run.ws,
+                                   run.status)
+        torch.cuda.synchronize()
+        assert int(run.status.item()) == 0
+        run.mem.check("attention at a full-size configuration")
     oc, lc = o[0].cpu(), lse[0].cpu()
 
     class View:
@@ -125,6 +130,70 @@ def test_hunyuan720p_sparse_and_dense():
     run, worst, ties = run_pipeline("hunyuan720p", 1024, expect=[8, 8, 8])
     Od, ld = gpu_outputs(run, dense=True)
     check_rows(run, Od, ld, [D_] * run.wl.H, synth.sample_rows(run.wl, 128, seed=5), [0, 9, 18, 23])
+
+
+BANDWIDTHS = [0.125, 0.25, 0.5]
+
+
+@pytest.mark.parametrize("name", ["opensoraplan", "hunyuan720p"])
+def test_dynamic_bandwidth_at_full_size(name):
+    """RainFusion+ (Sec. 4.3, last paragraph) at the two large shapes: every candidate's recalls, the (pattern,
+    window) each head takes, tile lists built from each head's own window, and 256 rows per head of the
+    attention that honours it, all against the oracle."""
+    wl = synth.WORKLOADS[name]
+    g = gu.geom(wl)
+    run = gu.Run(wl, qkv=inputs(name))
+    cls_gpu, win_gpu, rec_gpu = (x[0] for x in run.arm_plus(BANDWIDTHS))
+    chosen = set()
+    for h in range(wl.H):
+        cls, idx, window, Rt, Rs = orc.arm_head_plus(run.q_bits[0, h], run.k_bits[0, h], g, BANDWIDTHS, wl.textural_stride,
+                                                     wl.sample_mode, wl.sample_stride, wl.alpha)
+        assert np.abs(rec_gpu[h, 0] - np.asarray(Rt)).max() <= gu.RECALL_ABS, (h, rec_gpu[h, 0], Rt)
+        assert np.abs(rec_gpu[h, 1] - np.asarray(Rs)).max() <= gu.RECALL_ABS, (h, rec_gpu[h, 1], Rs)
+        if min(abs(r - wl.alpha) for r in list(Rt) + list(Rs)) > gu.TIE_MARGIN:
+            assert (int(cls_gpu[h]), int(win_gpu[h])) == (cls, window), h
+        chosen.add((int(cls_gpu[h]), int(win_gpu[h])))
+    assert {c for c, _ in chosen} == {S_, T_, X_}                  # the planted thirds still reach all three patterns
+    run.build_plus()
+
+    def pp_of_head(h):
+        c, w = int(cls_gpu[h]), int(win_gpu[h])
+        return orc.PatternParams(w if c == S_ else wl.frame_window, w if c == T_ else wl.spatial_window, wl.textural_stride)
+
+    tiles = sample_tiles(run.sched.nQ, k=4)
+    first = {}                                                     # (class, window) -> lists of the first such head
+    for h in range(wl.H):
+        key = (int(cls_gpu[h]), int(win_gpu[h]))
+        got = run.lists(0, h)
+        if key in first:                                           # same class and window: the lists must repeat
+            assert got == first[key], h
+            continue
+        first[key] = got
+        for a in tiles:
+            assert got[a] == orc.tile_row(key[0], g, pp_of_head(h), True, 128, 128, a), (name, h, a)
+        assert int(run.sched.kv_len[0, h]) == orc.kv_len(key[0], g, pp_of_head(h))
+    O, lse = gpu_outputs(run, plus=True)
+    check_rows(run, O, lse, cls_gpu, synth.sample_rows(wl, 256, seed=9), range(wl.H), pp_of_head)
+
+
+def test_two_mask_ablation_at_cogvideox_literal_amplitude():
+    """Table 2's rows without the Textural mask at the CogVideoX shape with the planted amplitude its configuration
+    states (0.5): neither recall reaches alpha for any head, so every head takes the mask of larger recall."""
+    wl = synth.WORKLOADS["cogvideox"]
+    run = gu.Run(wl, qkv=inputs("cogvideox"), two_mask=1)
+    cls_gpu, rec_gpu = run.arm()
+    cls_ref, rec_ref, margin = orc.arm_classify(run.q_bits, run.k_bits, gu.geom(wl), gu.pparams(wl), wl.sample_mode,
+                                                wl.sample_stride, wl.alpha, two_mask=True)
+    assert np.abs(rec_gpu - rec_ref).max() <= gu.RECALL_ABS
+    assert rec_ref[..., :2].max() < wl.alpha                       # the fallback branch decided every head
+    decided = margin > gu.TIE_MARGIN
+    assert np.array_equal(cls_gpu[decided], cls_ref[decided])
+    assert set(cls_gpu.reshape(-1).tolist()) <= {S_, T_} and X_ not in cls_ref
+    run.build()
+    classes = cls_gpu[0]
+    check_lists(run, classes, None)
+    O, lse = gpu_outputs(run)
+    check_rows(run, O, lse, classes, synth.sample_rows(wl, 256, seed=10), range(wl.H))
 
 
 @pytest.mark.parametrize("name", ["sweep_8x1024", "sweep_16x2040", "sweep_33x3600"])

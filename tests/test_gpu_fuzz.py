@@ -96,10 +96,11 @@ def test_random_case_dynamic_bandwidth(seed):
     bws = sorted(set(float(x) for x in rng.choice([0.05, 0.125, 0.2, 0.25, 0.4, 0.5, 0.75, 1.0], size=int(rng.integers(1, 5)))))
     g = gu.geom(wl)
     run = gu.Run(wl, temporal_permute=permute, two_mask=two_mask)
-    head_window = torch.full((wl.B, wl.H), -7, dtype=torch.int32, device="cuda")
-    rec = torch.zeros((wl.B, wl.H, 2, len(bws)), dtype=torch.float32, device="cuda")
-    api.rf_arm_classify_plus(run.shape, run.params, bws, run.q, run.k, run.head_class, head_window, rec, run.ws)
+    head_window = run.mem.alloc((wl.B, wl.H), torch.int32, -7, "head_window")
+    rec = run.mem.alloc((wl.B, wl.H, 2, len(bws)), torch.float32, 0, "recall_plus")
+    api.rf_arm_classify_plus(run.shape, run.params, bws, run.q, run.k, run.head_class, head_window, rec, run.ws, run.status)
     torch.cuda.synchronize()
+    run.mem.check("rf_arm_classify_plus")
     cls_gpu, win_gpu, rec_gpu = run.head_class.cpu().numpy(), head_window.cpu().numpy(), rec.cpu().numpy()
     for b in range(wl.B):
         for h in range(wl.H):
@@ -111,12 +112,12 @@ def test_random_case_dynamic_bandwidth(seed):
             if margin > gu.TIE_MARGIN:
                 assert (int(cls_gpu[b, h]), int(win_gpu[b, h])) == (cls, window), (seed, b, h)
     api.rf_build_block_mask_plus(run.shape, run.params, run.head_class, head_window, run.sched, run.status)
-    o = torch.full((wl.B, wl.H, wl.N, wl.D), float("nan"), dtype=torch.bfloat16, device="cuda")
-    lse = torch.full((wl.B, wl.H, wl.N), float("nan"), dtype=torch.float32, device="cuda")
+    o, lse = run.outputs()
     api.rf_sparse_attn_fwd_plus(run.shape, run.params, run.q, run.k, run.v, run.head_class, head_window, run.sched, o, lse,
                                 run.ws, run.status)
     torch.cuda.synchronize()
     assert int(run.status.item()) == 0
+    run.mem.check("rf_build_block_mask_plus / rf_sparse_attn_fwd_plus")
     O, LSE = o.float().cpu().numpy().astype(np.float64), lse.cpu().numpy().astype(np.float64)
     for b in range(wl.B):
         for h in range(wl.H):

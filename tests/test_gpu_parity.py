@@ -232,9 +232,9 @@ def test_boundary_spotlight_and_poison(cls, permute, inside):
     O, lse = run.sparse()
     Or, lr = orc.masked_attention(q, k, v, cls, gu.geom(wl), gu.pparams(wl))
     assert np.abs(Or).max() > 1.0                       # the planted keys matter for the reference
-    err = np.abs(O[0, 0] - Or)
-    assert err.max() <= 5e-2 * max(1.0, np.abs(Or).max()), err.max()
-    assert np.abs(lse[0, 0] - lr).max() <= 5e-3
+    # the stated bars (max-abs scaled per row by that row's own magnitude; lse 2e-3): a planted key dominates its
+    # rows, so the outputs are the planted values themselves and the measured errors are orders below the bars
+    gu.check_attention(O[0, 0], lse[0, 0], Or, lr, f"boundary class {cls} permute {permute} inside {inside}", strict=False)
 
 
 # ------------------------------------------------------------------ degenerate shapes and parameters
@@ -272,6 +272,30 @@ def test_arm_edge_shapes():
             check_arm(wl)
 
 
+def test_windows_and_stride_far_past_the_extent():
+    """frame_window, spatial_window and textural_stride at INT_MAX: the masks are those of the extent itself
+    (everything kept; the diagonal y == x), recalls 1, and nothing in the index arithmetic overflows."""
+    big = 2**31 - 1
+    for mode in (0, 1):
+        wl = synth.small_workload("huge_windows", H=3, D=64, T=5, fh=6, fw=7, L=3, mode=mode, omega=3, wf=big, ws=big, tau=big)
+        run = gu.Run(wl)
+        cls_gpu, cls_ref, _ = check_arm(wl, run)
+        assert cls_gpu.tolist() == [[T_] * 3]
+        assert np.abs(run.recall.cpu().numpy()[..., :2] - 1.0).max() <= gu.RECALL_ABS
+        run.force_classes([S_, T_, X_])
+        run.build()
+        for h, cls in enumerate([S_, T_, X_]):
+            ref = gu.oracle_lists(wl, cls, 128, 1)
+            assert run.lists(0, h) == [ref[a] for a in range(run.sched.nQ)]
+        O, lse = run.sparse()
+        for h, cls in enumerate([S_, T_, X_]):
+            Or, lr = orc.masked_attention(run.q_bits[0, h], run.k_bits[0, h], run.v_bits[0, h], cls, gu.geom(wl), gu.pparams(wl))
+            gu.check_attention(O[0, h], lse[0, h], Or, lr, f"huge windows class {cls}")
+            if cls != X_:
+                Od, ld = orc.masked_attention(run.q_bits[0, h], run.k_bits[0, h], run.v_bits[0, h], D_, gu.geom(wl), gu.pparams(wl))
+                assert np.array_equal(Or, Od)
+
+
 def test_scores_with_large_dynamic_range_do_not_overflow():
     """Logits that jump by far more than the lazy-rescale threshold between tiles, and rows whose first
     tiles are fully masked: the running maximum must be raised (and O rescaled) exactly."""
@@ -306,6 +330,37 @@ def test_bounded_wait_runs_out_cleanly_and_the_context_stays_usable():
     assert int(ret.item()) == 4               # neither wait succeeded; abort flag set
     assert 15.0 <= t0.elapsed_time(t1) <= 500.0
     test_dense_tiny()                         # the context is intact
+
+
+def test_arm_failure_is_reported_and_poisons_the_classes():
+    """ARM's reporting of a wait that ran out, exercised without making any wait run out: the self-test runs
+    rf_arm_classify's launch sequence with the score kernel's failure flag set in place of the kernel.  The
+    decision kernel must then write class -1 for every head and pass RF_ERR_TIMEOUT on; the tile builder and the
+    attention kernel, handed those classes, report them through their own status; a normal call afterwards
+    clears the flag and classifies as usual."""
+    wl = synth.WORKLOADS["tiny"]
+    run = gu.Run(wl)
+    cls_ok, _ = run.arm()
+    assert int(run.status.item()) == 0 and (cls_ok >= 0).all()
+    api.rf_selftest_arm_abandoned(run.shape, run.params, run.q, run.k, run.head_class, run.ws, run.status)
+    torch.cuda.synchronize()
+    assert int(run.status.item()) == 5                         # RF_ERR_TIMEOUT
+    assert run.head_class.cpu().numpy().tolist() == [[-1] * wl.H]
+    # a caller that gave ARM no status pointer still hears about it from the next stage
+    api.rf_selftest_arm_abandoned(run.shape, run.params, run.q, run.k, run.head_class, run.ws, None)
+    later = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.rf_build_block_mask(run.shape, run.params, run.head_class, run.sched, later)
+    torch.cuda.synchronize()
+    assert int(later.item()) == 1                              # RF_ERR_INVALID_ARG: class outside 0..3
+    later.zero_()
+    o = torch.empty_like(run.q)
+    api.rf_sparse_attn_fwd(run.shape, run.params, run.q, run.k, run.v, run.head_class, run.sched, o, None, run.ws, later)
+    torch.cuda.synchronize()
+    assert int(later.item()) == 1
+    # the flag is per call: the next real call classifies normally
+    run.status.zero_()
+    cls_again, _ = run.arm()
+    assert int(run.status.item()) == 0 and np.array_equal(cls_again, cls_ok)
 
 
 @pytest.mark.parametrize("D", [64, 96, 128])

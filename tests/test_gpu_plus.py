@@ -44,11 +44,7 @@ def test_dynamic_bandwidth_pipeline(mode):
     v = np.stack([h[2] for h in heads])[None]
     run = gu.Run(wl, qkv=(q, k, v))
     g = gu.geom(wl)
-    head_window = torch.full((wl.B, wl.H), -7, dtype=torch.int32, device="cuda")
-    rec = torch.zeros((wl.B, wl.H, 2, len(BWS)), dtype=torch.float32, device="cuda")
-    api.rf_arm_classify_plus(run.shape, run.params, BWS, run.q, run.k, run.head_class, head_window, rec, run.ws)
-    torch.cuda.synchronize()
-    cls_gpu, win_gpu, rec_gpu = run.head_class.cpu().numpy()[0], head_window.cpu().numpy()[0], rec.cpu().numpy()[0]
+    cls_gpu, win_gpu, rec_gpu = (x[0] for x in run.arm_plus(BWS))
 
     seen = set()
     for h in range(wl.H):
@@ -63,14 +59,8 @@ def test_dynamic_bandwidth_pipeline(mode):
     assert len(seen) >= 4          # the planted heads really exercise several (pattern, bandwidth) outcomes
 
     # schedule and attention with the per-head windows the GPU chose
-    api.rf_build_block_mask_plus(run.shape, run.params, run.head_class, head_window, run.sched, run.status)
-    o = torch.full((wl.B, wl.H, wl.N, wl.D), float("nan"), dtype=torch.bfloat16, device="cuda")
-    lse = torch.full((wl.B, wl.H, wl.N), float("nan"), dtype=torch.float32, device="cuda")
-    api.rf_sparse_attn_fwd_plus(run.shape, run.params, run.q, run.k, run.v, run.head_class, head_window, run.sched, o, lse,
-                                run.ws, run.status)
-    torch.cuda.synchronize()
-    assert int(run.status.item()) == 0
-    O, LSE = o.float().cpu().numpy().astype(np.float64)[0], lse.cpu().numpy().astype(np.float64)[0]
+    run.build_plus()
+    O, LSE = (x[0] for x in run.sparse_plus())
     for h in range(wl.H):
         cls, w = int(cls_gpu[h]), int(win_gpu[h])
         pp = orc.PatternParams(w if cls == orc.SPATIAL else wl.frame_window, w if cls == orc.TEMPORAL else wl.spatial_window,
@@ -90,11 +80,7 @@ def test_dynamic_bandwidth_with_two_masks():
              synth.make_head(wl, 0, 4, kind="lowrank"), synth.make_head(wl, 0, 5, kind="none")]
     q, k, v = (np.stack([h[i] for h in heads])[None] for i in range(3))
     run = gu.Run(wl, qkv=(q, k, v), two_mask=1)
-    head_window = torch.full((wl.B, wl.H), -7, dtype=torch.int32, device="cuda")
-    rec = torch.zeros((wl.B, wl.H, 2, len(BWS)), dtype=torch.float32, device="cuda")
-    api.rf_arm_classify_plus(run.shape, run.params, BWS, run.q, run.k, run.head_class, head_window, rec, run.ws)
-    torch.cuda.synchronize()
-    cls_gpu, win_gpu = run.head_class.cpu().numpy()[0], head_window.cpu().numpy()[0]
+    cls_gpu, win_gpu, _ = (x[0] for x in run.arm_plus(BWS))
     g = gu.geom(wl)
     fell_back = 0
     for h in range(wl.H):

@@ -48,6 +48,35 @@ def test_two_gloo_ranks_take_the_max_and_sum_the_replicas():
         assert abs(thr - 2 * 1e3 / 15e-3) < 1e-6
 
 
+def test_bare_bench_command_with_gpus_2_starts_two_replicas():
+    """`python bench.py --gpus 2` without a launcher spawns its own two ranks (gloo and a stub step here): rank 0
+    prints one line whose n_gpus is 2 and whose time is the slower rank's."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--stub", "--workload", "tiny",
+                        "--steps", "3", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    lines = [l for l in r.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["config"]["parallelism"] == "replicas x2"
+    assert line["ms_per_step"] >= 19.0             # rank 1 sleeps 20 ms per step, rank 0 only 10
+    # under a launcher (WORLD_SIZE set) a mismatching --gpus is an error, not a silent single replica
+    env2 = dict(env, RANK="0", WORLD_SIZE="1", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--stub", "--workload", "tiny"],
+                       env=env2, capture_output=True, text=True, timeout=300)
+    assert r.returncode != 0 and "WORLD_SIZE" in r.stderr
+
+
+def test_a_failing_rank_ends_the_launcher_with_its_code():
+    sys.path.insert(0, ROOT)
+    from paper_2505_21036_b200 import dist_util
+    prog = "import os, sys, time; r = int(os.environ['RANK']); sys.exit(7) if r == 1 else time.sleep(60)"
+    import time
+    t0 = time.time()
+    assert dist_util.spawn_replicas([sys.executable, "-c", prog], 2) == 7
+    assert time.time() - t0 < 30.0                  # rank 0 was not left sleeping
+
+
 def test_single_rank_is_identity():
     sys.path.insert(0, ROOT)
     from paper_2505_21036_b200 import dist_util

@@ -58,6 +58,6 @@ def test_noalloc_rejects_problems_beyond_its_scratch():
     big = api.make_shape(4, 64, 128, 33, 45, 80, 256)
     params = api.make_params(8, 900, sample_stride=36)
     # the pointers are never dereferenced: the size check comes before any CUDA call
-    code = api.load().rf_arm_classify_noalloc(big, params, 16, 16, 16, None, None)
+    code = api.load().rf_arm_classify_noalloc(big, params, 16, 16, 16, None, None, None)
     assert code == 6          # RF_ERR_STATIC_SCRATCH_TOO_SMALL
     assert b"built-in" in api.load().rf_status_string(code)

@@ -15,13 +15,13 @@
 // from TMEM.  The running maximum is raised lazily (see kSumLimit), in which case the softmax warp itself
 // rescales its rows of O in TMEM; the final O / l and the log-sum-exp do not depend on it.
 // PARTIAL tiles apply the exact element mask of the head's pattern; FULL tiles skip it.
-#include "rf_sm100.cuh"
+#include "rf_attn_common.cuh"
 
 namespace {
 
 using namespace sm100;
+using namespace rf_attn;
 
-constexpr int BM = 128, BN = 128;
 constexpr int kThreads = kWsThreads;        // 3 warpgroups: softmax 0, softmax 1, {TMA, MMA, 2 idle warps}
 constexpr int kTmaWarp = 8, kMmaWarp = 9;
 // Lazy rescaling of the running maximum.  A tile's weights are taken as 2^(score - running maximum) and accepted
@@ -72,135 +72,6 @@ struct Cfg {
   // TMEM columns
   static constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL0 = 256, O_COL1 = S_EARLY ? 320 : 384, TMEM_COLS = 512;
   static constexpr uint32_t P_COL0 = S_EARLY ? 384 : S_COL0, P_COL1 = S_EARLY ? 448 : S_COL1;   // packed bf16, 64 columns
-};
-
-// The two bf16 values of a packed word, widened exactly.  The row sum is taken over these rounded weights, the
-// ones the tensor core multiplies with V: O / l is then an exact convex combination of V rows with slightly
-// perturbed weights, and the rounding of a dominant weight cancels instead of scaling the whole output row.
-__device__ __forceinline__ float2 unpack_bf16(uint32_t w) {
-  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// Element mask of one query row in the head's key-slot space, evaluated per tile as a 128-bit word
-// (bit c = key slot u0 + c kept).  Every pattern's kept set is a union of a few slot intervals:
-// one window [lo, hi) (Spatial, position-major Temporal), one band per frame (Temporal in original
-// order) and the always-kept text slots [text0, lkv).  Kept compact on purpose: PARTIAL tiles are
-// rare, and a large rarely-run code block costs more in instruction fetch than in arithmetic.
-struct RowMask {
-  int lo, hi;        // kept video slots [lo, hi) when !periodic
-  int text0;         // first always-kept (text) slot
-  int lkv;           // number of key slots
-  int p, ws, S, T;   // periodic form: |slot % S - p| <= ws for slots of frames 0..T-1
-  bool periodic;
-
-  static __device__ __forceinline__ uint32_t below(int n) {  // bits [0, n) set, n in [0, 32]
-    return n >= 32 ? 0xffffffffu : ((1u << n) - 1u);
-  }
-  // OR the slots [a, b) (absolute) into the tile's words.
-  static __device__ __forceinline__ void add(uint32_t (&w)[4], int u0, int a, int b) {
-    a = max(a - u0, 0);
-    b = min(b - u0, BN);
-    if (a >= b) return;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int lo_k = min(max(a - 32 * k, 0), 32), hi_k = min(max(b - 32 * k, 0), 32);
-      w[k] |= below(hi_k) & ~below(lo_k);
-    }
-  }
-  __device__ __noinline__ void tile_bits(int u0, uint32_t (&w)[4]) const {
-    w[0] = w[1] = w[2] = w[3] = 0u;
-    if (periodic) {
-      const int f1 = min((u0 + BN - 1) / S, T - 1);
-      for (int f = u0 / S; f <= f1; ++f) add(w, u0, f * S + max(p - ws, 0), f * S + min(p + ws, S - 1) + 1);
-    } else {
-      add(w, u0, lo, min(hi, text0));
-    }
-    add(w, u0, text0, lkv);
-  }
-};
-
-__device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r) {
-  RowMask m;
-  m.lkv = rf_kv_len(g, cls);
-  m.text0 = m.lkv;
-  m.lo = 0;
-  m.hi = m.lkv;
-  m.p = 0; m.ws = g.ws; m.S = g.S; m.T = g.T;
-  m.periodic = false;
-  if ((cls == RF_SPATIAL || cls == RF_TEMPORAL) && r < g.Nv) {
-    m.text0 = g.Nv;
-    if (cls == RF_SPATIAL) {
-      const int f = r / g.S;
-      m.lo = max(0, f - g.wf) * g.S;
-      m.hi = min(g.T, f + g.wf + 1) * g.S;
-    } else if (g.permute) {
-      const int p = r / g.T;
-      m.lo = max(0, p - g.ws) * g.T;
-      m.hi = min(g.S, p + g.ws + 1) * g.T;
-    } else {
-      m.periodic = true;
-      m.p = r % g.S;
-    }
-  }
-  return m;
-}
-
-// Exact maximum of this thread's row of the S tile at t_s (slow path of the softmax; warp-collective loads).
-__device__ __noinline__ float tile_row_max(uint32_t t_s, bool partial, const RowMask& rmask, int u0) {
-  uint32_t w[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
-  if (partial) rmask.tile_bits(u0, w);
-  float mx = -INFINITY;
-#pragma unroll 1
-  for (int q = 0; q < 4; ++q) {
-    uint32_t v[32];
-    tmem_ld32(t_s + q * 32, v);
-    tc_wait_ld();
-#pragma unroll
-    for (int c = 0; c < 32; ++c)
-      if ((w[q] >> c) & 1u) mx = fmaxf(mx, __uint_as_float(v[c]));
-  }
-  return mx;
-}
-
-// The two streams' ascending tile lists and their merge (the order K/V tiles are fetched in).
-struct Lists {
-  const int32_t* l0;
-  const int32_t* l1;
-  int n0, n1;
-  int lkv;
-  bool listed;
-  __device__ __forceinline__ uint32_t entry(int j, int i) const {
-    if (listed) return (uint32_t)(j == 0 ? l0[i] : l1[i]);
-    const bool tail = (i + 1) * BN > lkv;
-    return (uint32_t)i | (tail ? RF_PARTIAL_BIT : 0u);
-  }
-};
-struct Merge {
-  int i0 = 0, i1 = 0;
-  // Raw list entries at i0 / i1, loaded by the previous call and not touched until the next one, so
-  // that the load latency never sits between two MMA bursts of the (in-order) issuing thread.
-  uint32_t raw0 = 0, raw1 = 0;
-  __device__ __forceinline__ void start(const Lists& L) {
-    if (L.n0 > 0) raw0 = L.entry(0, 0);
-    if (L.n1 > 0) raw1 = L.entry(1, 0);
-  }
-  // Next tile of the union; uses bit j set when stream j lists it.  Returns false when exhausted.
-  __device__ __forceinline__ bool next(const Lists& L, int& tile, int& uses) {
-    const int h0 = i0 < L.n0 ? (int)(raw0 & ~RF_PARTIAL_BIT) : 0x7fffffff;
-    const int h1 = i1 < L.n1 ? (int)(raw1 & ~RF_PARTIAL_BIT) : 0x7fffffff;
-    tile = min(h0, h1);
-    if (tile == 0x7fffffff) return false;
-    uses = (h0 == tile ? 1 : 0) | (h1 == tile ? 2 : 0);
-    if ((uses & 1) && ++i0 < L.n0) raw0 = L.entry(0, i0);
-    if ((uses & 2) && ++i1 < L.n1) raw1 = L.entry(1, i1);
-    return true;
-  }
 };
 
 template <int D>

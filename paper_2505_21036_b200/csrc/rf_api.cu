@@ -1,6 +1,5 @@
 // C ABI of the RainFusion CUDA path: argument validation, workspace layout, tensor-map encoding.
 #include <math.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include "rf_common.cuh"
@@ -91,8 +90,8 @@ EncodeTiledFn encode_fn() {
 }
 
 // bf16 [heads][rows (stride head_rows)][D] viewed as a 3-D tensor, box = 64 columns x 128 rows, 128B swizzle.
-bool encode_map(CUtensorMap* m, const void* ptr, int D, int rows, int head_rows, int heads, int box_rows = 128) {
-  return rf_encode_rows_map(m, ptr, D, rows, (size_t)D * 2, (size_t)head_rows * D * 2, heads, box_rows);
+bool encode_map(CUtensorMap* m, const void* ptr, int D, int rows, int head_rows, int heads) {
+  return rf_encode_rows_map(m, ptr, D, rows, (size_t)D * 2, (size_t)head_rows * D * 2, heads);
 }
 
 rf_status check_attn_shape(const rf_shape* s) {
@@ -104,22 +103,13 @@ rf_status check_attn_shape(const rf_shape* s) {
 
 }  // namespace
 
-bool rf_use_pair_kernel() {
-  static int choice = -1;
-  if (choice < 0) {
-    const char* e = getenv("RF_ATTN_KERNEL");
-    choice = (e != nullptr && strcmp(e, "pair") == 0) ? 1 : 0;
-  }
-  return choice == 1;
-}
-
 bool rf_encode_rows_map(CUtensorMap* m, const void* ptr, int D, int rows, size_t row_stride_bytes,
-                        size_t head_stride_bytes, int heads, int box_rows) {
+                        size_t head_stride_bytes, int heads) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)heads};
   cuuint64_t strides[2] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)head_stride_bytes};
-  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t box[3] = {64, 128, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -167,9 +157,7 @@ rf_status sparse_attn_impl(const rf_shape* shape, const rf_params* params, const
   bool ok = encode_map(&maps[0], q, g.D, g.N, g.N, heads) && encode_map(&maps[1], k, g.D, g.N, g.N, heads) &&
             encode_map(&maps[2], v, g.D, g.N, g.N, heads) && encode_map(&maps[3], wq, g.D, g.N, g.N, heads) &&
             encode_map(&maps[4], wk, g.D, g.N, g.N, heads) && encode_map(&maps[5], wv, g.D, g.N, g.N, heads) &&
-            encode_map(&maps[6], wk, g.D, g.LkvTex, g.N, heads) && encode_map(&maps[7], wv, g.D, g.LkvTex, g.N, heads) &&
-            encode_map(&maps[8], k, g.D, g.N, g.N, heads, 64) && encode_map(&maps[9], wk, g.D, g.N, g.N, heads, 64) &&
-            encode_map(&maps[10], wk, g.D, g.LkvTex, g.N, heads, 64);
+            encode_map(&maps[6], wk, g.D, g.LkvTex, g.N, heads) && encode_map(&maps[7], wv, g.D, g.LkvTex, g.N, heads);
   if (!ok) return RF_ERR_CUDA;
 
   if (gather) {
@@ -189,7 +177,7 @@ rf_status sparse_attn_impl(const rf_shape* shape, const rf_params* params, const
   a.lse = lse;
   a.dev_status = dev_status;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.D);
-  return rf_use_pair_kernel() ? rf_launch_attention_pair(a, maps, stream) : rf_launch_attention(a, maps, stream);
+  return rf_launch_attention(a, maps, stream);
 }
 }  // namespace
 
@@ -373,10 +361,9 @@ rf_status rf_dense_attn_fwd(const rf_shape* shape, const void* q, const void* k,
   CUtensorMap maps[RF_ATTN_MAPS];
   const int heads = g.B * g.H;
   bool ok = encode_map(&maps[0], q, g.D, g.N, g.N, heads) && encode_map(&maps[1], k, g.D, g.N, g.N, heads) &&
-            encode_map(&maps[2], v, g.D, g.N, g.N, heads) && encode_map(&maps[8], k, g.D, g.N, g.N, heads, 64);
+            encode_map(&maps[2], v, g.D, g.N, g.N, heads);
   if (!ok) return RF_ERR_CUDA;
   for (int i = 3; i < 8; ++i) maps[i] = maps[i % 3];
-  maps[9] = maps[10] = maps[8];
   RfAttnArgs a;
   a.g = g;
   a.head_class = nullptr;
@@ -387,8 +374,7 @@ rf_status rf_dense_attn_fwd(const rf_shape* shape, const void* q, const void* k,
   a.lse = lse;
   a.dev_status = dev_status;
   a.scale_log2 = 1.4426950408889634f / sqrtf((float)g.D);
-  return rf_use_pair_kernel() ? rf_launch_attention_pair(a, maps, static_cast<cudaStream_t>(cuda_stream))
-                              : rf_launch_attention(a, maps, static_cast<cudaStream_t>(cuda_stream));
+  return rf_launch_attention(a, maps, static_cast<cudaStream_t>(cuda_stream));
 }
 
 }  // extern "C"

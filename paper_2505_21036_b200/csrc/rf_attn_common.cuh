@@ -17,40 +17,10 @@ __device__ __forceinline__ float2 unpack_bf16(uint32_t w) {
   return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }
 
-// acc += the two bf16 values of a packed word, widened exactly (mixed-precision adds: no unpacking)
-__device__ __forceinline__ void add_bf16x2(float& acc_lo, float& acc_hi, uint32_t w) {
-  asm("{\n\t.reg .b16 lo, hi;\n\t"
-      "mov.b32 {lo, hi}, %2;\n\t"
-      "add.rn.f32.bf16 %0, lo, %0;\n\t"
-      "add.rn.f32.bf16 %1, hi, %1;\n\t}"
-      : "+f"(acc_lo), "+f"(acc_hi)
-      : "r"(w));
-}
-
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-
-// 2^x for two values on the FMA pipe: the MUFU unit takes 16 exponentials per clock and SM, which at head dimension
-// 128 costs as many cycles per tile as the tensor cores' two contractions; part of the exponentials therefore runs
-// as round-to-nearest range reduction (magic-number add) plus a degree-3 minimax polynomial on [-1/2, 1/2]
-// (max relative error 7.6e-5, far inside the bf16 rounding of P) and an integer add into the exponent field.
-// Inputs below -126 (masked scores are -inf) give 2^-126.
-__device__ __forceinline__ float2 ex2_poly2(float2 x) {
-  x.x = fmaxf(x.x, -126.f);
-  x.y = fmaxf(x.y, -126.f);
-  const float2 magic = make_float2(12582912.f, 12582912.f);                  // 1.5 * 2^23: low mantissa bits = round(x)
-  const float2 y = __fadd2_rn(x, magic);
-  const float2 n = __fadd2_rn(y, make_float2(-12582912.f, -12582912.f));
-  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-  float2 p = __ffma2_rn(f, make_float2(0.05520550534129143f, 0.05520550534129143f), make_float2(0.24261397123336792f, 0.24261397123336792f));
-  p = __ffma2_rn(p, f, make_float2(0.6932547688484192f, 0.6932547688484192f));
-  p = __ffma2_rn(p, f, make_float2(0.9999276995658875f, 0.9999276995658875f));
-  p.x = __int_as_float(__float_as_int(y.x) * (1 << 23) + __float_as_int(p.x));   // one integer multiply-add per value
-  p.y = __int_as_float(__float_as_int(y.y) * (1 << 23) + __float_as_int(p.y));
-  return p;
 }
 
 // Element mask of one query row in the head's key-slot space, evaluated per tile as a 128-bit word

@@ -58,7 +58,7 @@ size_t rf_arm_scratch_floats(const RfGeom& g, int omega, int nb);
 // Tensor map over bf16 rows: [heads][rows][D] with the given row and head strides in bytes (multiples of 16),
 // box = 64 columns x 128 rows, 128-byte swizzle, zero fill past `rows`.
 bool rf_encode_rows_map(CUtensorMap* m, const void* ptr, int D, int rows, size_t row_stride_bytes,
-                        size_t head_stride_bytes, int heads, int box_rows = 128);
+                        size_t head_stride_bytes, int heads);
 // Validates shape and parameters as the entry points do and fills the kernel-side geometry.
 rf_status rf_checked_geom(const rf_shape* shape, const rf_params* params, RfGeom* out);
 
@@ -74,12 +74,7 @@ struct RfAttnArgs {
   float scale_log2;           // log2(e) / sqrt(D)
 };
 // Tensor maps: [0..2] Q/K/V in original order, [3..5] the workspace copies with N rows per head
-// (position-major Q/K/V of Temporal heads), [6..7] workspace K/V with LkvTex rows per head (Textural);
-// [8..10] K once more with 64-row boxes for the CTA-pair kernel (original, position-major, compacted).
-constexpr int RF_ATTN_MAPS = 11;
+// (position-major Q/K/V of Temporal heads), [6..7] workspace K/V with LkvTex rows per head (Textural).
+constexpr int RF_ATTN_MAPS = 8;
 rf_status rf_launch_attention(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st);
-rf_status rf_launch_attention_pair(const RfAttnArgs& a, const CUtensorMap* maps, cudaStream_t st);
-// Which of the two attention kernels a call runs: the single-CTA kernel unless the environment variable
-// RF_ATTN_KERNEL says "pair" (read once per process; for A/B measurements).
-bool rf_use_pair_kernel();
 rf_status rf_launch_selftest_timeout(int32_t* dev_status, uint64_t limit_ns, int32_t* waits_returned, cudaStream_t st);

@@ -46,7 +46,9 @@ typedef enum {
   RF_ERR_WORKSPACE_TOO_SMALL = 3,
   RF_ERR_CUDA = 4,
   RF_ERR_TIMEOUT = 5,
-  RF_ERR_STATIC_SCRATCH_TOO_SMALL = 6
+  RF_ERR_STATIC_SCRATCH_TOO_SMALL = 6,
+  RF_ERR_BOUNDS = 7   /* only from a library built with -DRF_BOUNDS_CHECK: a kernel was about to index outside an
+                         array (reported through dev_status; the access is skipped, nothing traps) */
 } rf_status;
 
 /* Head categories (Sec. 3.2).  RF_DENSE is not an ARM outcome; a caller may force it. */
@@ -96,6 +98,11 @@ typedef struct {
 } rf_schedule;
 
 const char *rf_status_string(rf_status s);
+
+/* 1 if this library was built with -DRF_BOUNDS_CHECK (every kernel checks the indices of its global-memory
+ * writes and of the schedule entries it reads, reports RF_ERR_BOUNDS through dev_status and skips the access),
+ * else 0.  The memory checker of the CUDA toolkit is not available everywhere; this build is its stand-in for tests. */
+int32_t rf_bounds_checked(void);
 
 /* Host, pure: nQ = ceil(N/block_m), nKmax = ceil(N/block_n). */
 rf_status rf_schedule_dims(const rf_shape *shape, const rf_params *params, int32_t *nQ, int32_t *nKmax);

@@ -14,13 +14,15 @@ RF_SPATIAL, RF_TEMPORAL, RF_TEXTURAL, RF_DENSE = 0, 1, 2, 3
 RF_SAMPLE_ALG1, RF_SAMPLE_GLOBAL = 0, 1
 PARTIAL_BIT = 1 << 31
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librainfusion.so")
+# RAINFUSION_LIBRARY selects another build of the same library (the bounds-checking build, say); there is still no
+# fallback of any kind: the named file must exist and export every entry point.
+_LIB_PATH = os.environ.get("RAINFUSION_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "librainfusion.so")
 _lib = None
 
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
            "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
            "rf_arm_classify_noalloc", "rf_selftest_wait_timeout", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus",
-           "rf_sparse_attn_reordered", "rf_selftest_arm_abandoned"]
+           "rf_sparse_attn_reordered", "rf_selftest_arm_abandoned", "rf_bounds_checked"]
 
 
 class rf_shape(C.Structure):
@@ -56,6 +58,8 @@ def load():
         raise RainFusionError(f"{_LIB_PATH} is missing: build it with `python -m paper_2505_21036_b200.build`")
     lib = C.CDLL(_LIB_PATH)
     P, V, I, Z = C.POINTER, C.c_void_p, C.c_int, C.c_size_t
+    lib.rf_bounds_checked.restype = C.c_int32
+    lib.rf_bounds_checked.argtypes = []
     lib.rf_status_string.restype = C.c_char_p
     lib.rf_status_string.argtypes = [I]
     lib.rf_schedule_dims.restype = I

@@ -1,4 +1,8 @@
-"""Builds librainfusion.so (sm_100a) in-tree with nvcc.  `python -m paper_2505_21036_b200.build`."""
+"""Builds librainfusion.so (sm_100a) in-tree with nvcc.  `python -m paper_2505_21036_b200.build`.
+
+`--checked` builds librainfusion_checked.so as well: the same sources with -DRF_BOUNDS_CHECK, whose kernels check
+the indices of their global-memory writes and of the schedule they read (see rf_bounds_checked in the header).
+Select it with the environment variable RAINFUSION_LIBRARY=<path> (read by api.load)."""
 from __future__ import annotations
 
 import os
@@ -9,6 +13,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "librainfusion.so")
+LIB_CHECKED = os.path.join(PKG, "librainfusion_checked.so")
 SOURCES = ["rf_api.cu", "rf_mask.cu", "rf_arm.cu", "rf_attn.cu"]
 HEADERS = ["rf_common.cuh", "rf_sm100.cuh", "rf_attn_common.cuh", os.path.join("..", "..", "include", "rainfusion.h")]
 
@@ -20,19 +25,22 @@ def nvcc_path() -> str:
     return cand
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
+def stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, s) for s in SOURCES + HEADERS] + [os.path.abspath(__file__)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not stale():
-        return LIB
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    lib = LIB_CHECKED if checked else LIB
+    if not force and not stale(lib):
+        return lib
     cmd = [nvcc_path(), "-shared", "-Xcompiler", "-fPIC", "-O3", "-std=c++17", "-lineinfo",
-           "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB]
+           "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib]
+    if checked:
+        cmd += ["-DRF_BOUNDS_CHECK"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
@@ -41,8 +49,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     if verbose:
         print(res.stderr)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--checked" in sys.argv:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked=True))

@@ -163,7 +163,7 @@ rf_status sparse_attn_impl(const rf_shape* shape, const rf_params* params, const
   if (gather) {
     cudaError_t e = rf_launch_gather(g, head_class, static_cast<const __nv_bfloat16*>(q),
                                      static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), wq, wk, wv,
-                                     stream);
+                                     dev_status, stream);
     if (e != cudaSuccess) return RF_ERR_CUDA;
   }
 
@@ -183,6 +183,14 @@ rf_status sparse_attn_impl(const rf_shape* shape, const rf_params* params, const
 
 extern "C" {
 
+int32_t rf_bounds_checked(void) {
+#ifdef RF_BOUNDS_CHECK
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 const char* rf_status_string(rf_status s) {
   switch (s) {
     case RF_OK: return "ok";
@@ -193,6 +201,7 @@ const char* rf_status_string(rf_status s) {
     case RF_ERR_TIMEOUT: return "device-side wait timed out";
     case RF_ERR_STATIC_SCRATCH_TOO_SMALL:
       return "problem needs more scratch than the library's built-in array holds (use the workspace entry point)";
+    case RF_ERR_BOUNDS: return "a kernel of the bounds-checking build was about to index outside an array";
   }
   return "unknown status";
 }
@@ -344,7 +353,7 @@ rf_status rf_reorder_tokens(const rf_shape* shape, const rf_params* params, cons
   cudaError_t e = rf_launch_gather(g, head_class, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
                                    static_cast<const __nv_bfloat16*>(v), reinterpret_cast<__nv_bfloat16*>(w),
                                    reinterpret_cast<__nv_bfloat16*>(w + tensor_bytes(g)),
-                                   reinterpret_cast<__nv_bfloat16*>(w + 2 * tensor_bytes(g)),
+                                   reinterpret_cast<__nv_bfloat16*>(w + 2 * tensor_bytes(g)), nullptr,
                                    static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? RF_OK : RF_ERR_CUDA;
 }

@@ -335,7 +335,8 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
 #pragma unroll
         for (int k = 0; k < NM; ++k) {
           const bool is_t = k < NB, is_x = k == 2 * NB;
-          if (is_x ? TEX : (is_t ? sm.want_t != 0 : sm.want_s != 0)) out[(size_t)k * n_pad + m] = l_m[k] * inv;
+          if ((is_x ? TEX : (is_t ? sm.want_t != 0 : sm.want_s != 0)) && rf_in_bounds(m, n_pad, arm_flag))
+            out[(size_t)k * n_pad + m] = l_m[k] * inv;
         }
       }
     }

@@ -118,6 +118,9 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
   if (L.listed) {
     L.n0 = a.count[(size_t)bh * g.nQ + qt0];
     L.n1 = qt1 < g.nQ ? a.count[(size_t)bh * g.nQ + qt1] : 0;
+    // a schedule that was not built for this shape could hold any count: the checking build refuses to walk past a row
+    if (!rf_in_bounds(L.n0, g.nKmax + 1, a.dev_status)) L.n0 = 0;
+    if (!rf_in_bounds(L.n1, g.nKmax + 1, a.dev_status)) L.n1 = 0;
     L.l0 = a.kv_tile + ((size_t)bh * g.nQ + qt0) * g.nKmax;
     L.l1 = a.kv_tile + ((size_t)bh * g.nQ + min(qt1, g.nQ - 1)) * g.nKmax;
   } else {
@@ -500,7 +503,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
         uint32_t v[32];
         tmem_ld32(t_o + c * 32, v);   // warp-collective: rows past N take part, they just do not store
         tc_wait_ld();
-        if (r < g.N) {
+        if (r < g.N && rf_in_bounds(tok, g.N, a.dev_status)) {
 #pragma unroll
           for (int i = 0; i < 32; i += 8) {
             uint4 w;
@@ -512,7 +515,7 @@ __global__ void __launch_bounds__(kThreads, 1) rf_attn_kernel(const __grid_const
           }
         }
       }
-      if (r < g.N && a.lse != nullptr) a.lse[(size_t)bh * g.N + tok] = (m_run + log2f(l_exact)) * 0.6931471805599453f;
+      if (r < g.N && a.lse != nullptr && rf_in_bounds(tok, g.N, a.dev_status)) a.lse[(size_t)bh * g.N + tok] = (m_run + log2f(l_exact)) * 0.6931471805599453f;
     }
   }
 

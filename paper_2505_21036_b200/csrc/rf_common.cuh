@@ -28,6 +28,18 @@ __device__ __forceinline__ void rf_report(int32_t* dev_status, int code) {
   if (dev_status != nullptr) atomicCAS(dev_status, 0, code);
 }
 
+// Index check of the bounds-checking build: true when idx < limit; otherwise RF_ERR_BOUNDS is reported and the
+// caller skips the access.  Compiles to `true` in the normal build.
+#ifdef RF_BOUNDS_CHECK
+__device__ __forceinline__ bool rf_in_bounds(unsigned long long idx, unsigned long long limit, int32_t* dev_status) {
+  if (idx < limit) return true;
+  rf_report(dev_status, RF_ERR_BOUNDS);
+  return false;
+}
+#else
+__device__ __forceinline__ bool rf_in_bounds(unsigned long long, unsigned long long, int32_t*) { return true; }
+#endif
+
 __host__ __device__ __forceinline__ int rf_cdiv(int a, int b) { return (a + b - 1) / b; }
 
 // Number of key slots of a head of class `cls`.
@@ -41,7 +53,7 @@ cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, co
                                   int32_t* kv_tile, uint32_t* bitmap, int32_t* kv_len, int32_t* dev_status, cudaStream_t st);
 cudaError_t rf_launch_gather(const RfGeom& g, const int32_t* head_class, const __nv_bfloat16* q,
                              const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* wq, __nv_bfloat16* wk,
-                             __nv_bfloat16* wv, cudaStream_t st);
+                             __nv_bfloat16* wv, int32_t* dev_status, cudaStream_t st);
 // nb candidate windows per pattern (ws_list for Temporal, wf_list for Spatial, ascending).  head_window == nullptr:
 // plain Algorithm 1 on the first candidate (recall: [B,H,3] or null).  Otherwise dynamic bandwidth: head_window
 // receives each head's chosen window, recall_plus ([B,H,2,nb] or null) the candidates' recalls.

@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int
   }
   const int Lkv = rf_kv_len(g, cls);
   const int nK = rf_cdiv(Lkv, g.BN);
-  if (a == 0 && lane == 0) kv_len[bh] = Lkv;
+  if (a == 0 && lane == 0 && rf_in_bounds(bh, (size_t)g.B * g.H, dev_status)) kv_len[bh] = Lkv;
   int32_t* row = kv_tile + ((size_t)bh * g.nQ + a) * g.nKmax;
   const int words = rf_cdiv(g.nKmax, 32);
   uint32_t* brow = bitmap ? bitmap + ((size_t)bh * g.nQ + a) * words : nullptr;
@@ -91,11 +91,14 @@ __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int
     const int b = b0 + lane;
     const int f = (b < nK) ? tile_flag(g, cls, a, b) : 0;
     const unsigned m = __ballot_sync(0xffffffffu, f != 0);
-    if (brow && lane == 0) brow[b0 >> 5] = m;
-    if (f != 0) row[base + __popc(m & ((1u << lane) - 1))] = (int32_t)((uint32_t)b | (f == 1 ? RF_PARTIAL_BIT : 0u));
+    if (brow && lane == 0 && rf_in_bounds(b0 >> 5, words, dev_status)) brow[b0 >> 5] = m;
+    if (f != 0) {
+      const int slot = base + __popc(m & ((1u << lane) - 1));
+      if (rf_in_bounds(slot, g.nKmax, dev_status)) row[slot] = (int32_t)((uint32_t)b | (f == 1 ? RF_PARTIAL_BIT : 0u));
+    }
     base += __popc(m);
   }
-  if (lane == 0) count[(size_t)bh * g.nQ + a] = base;
+  if (lane == 0 && rf_in_bounds((size_t)bh * g.nQ + a, (size_t)g.B * g.H * g.nQ, dev_status)) count[(size_t)bh * g.nQ + a] = base;
 }
 
 // Reordered copies for heads whose coordinate space is not the original one.
@@ -105,7 +108,7 @@ __global__ void __launch_bounds__(256) rf_build_tiles_kernel(RfGeom g, const int
 __global__ void __launch_bounds__(256) rf_gather_kernel(RfGeom g, const int32_t* __restrict__ head_class,
                                                          const uint4* __restrict__ q, const uint4* __restrict__ k,
                                                          const uint4* __restrict__ v, uint4* __restrict__ wq,
-                                                         uint4* __restrict__ wk, uint4* __restrict__ wv) {
+                                                         uint4* __restrict__ wk, uint4* __restrict__ wv, int32_t* dev_status) {
   extern __shared__ int row_start[];  // [Hf] rank of the first kept token of each frame row (Textural)
   const int bh = blockIdx.y;
   const int cls = head_class[bh];
@@ -142,6 +145,7 @@ __global__ void __launch_bounds__(256) rf_gather_kernel(RfGeom g, const int32_t*
         dst = f * g.nC + row_start[y] + x / g.tau;
       }
     }
+    if (!rf_in_bounds(dst, perm ? g.N : g.LkvTex, dev_status)) continue;
     const size_t s = head_off + (size_t)i * vec + c, d = head_off + (size_t)dst * vec + c;
     if (perm) wq[d] = q[s];
     wk[d] = k[s];
@@ -160,13 +164,13 @@ cudaError_t rf_launch_build_tiles(const RfGeom& g, const int32_t* head_class, co
 
 cudaError_t rf_launch_gather(const RfGeom& g, const int32_t* head_class, const __nv_bfloat16* q,
                              const __nv_bfloat16* k, const __nv_bfloat16* v, __nv_bfloat16* wq, __nv_bfloat16* wk,
-                             __nv_bfloat16* wv, cudaStream_t st) {
+                             __nv_bfloat16* wv, int32_t* dev_status, cudaStream_t st) {
   const int vec = g.D / 8;
   const int rows_per_cta = 256 / vec;
   int gx = rf_cdiv(g.N, rows_per_cta);
   if (gx > 148 * 8) gx = 148 * 8;
   dim3 grid(gx, g.B * g.H);
   rf_gather_kernel<<<grid, 256, g.Hf * sizeof(int), st>>>(g, head_class, (const uint4*)q, (const uint4*)k,
-                                                           (const uint4*)v, (uint4*)wq, (uint4*)wk, (uint4*)wv);
+                                                           (const uint4*)v, (uint4*)wq, (uint4*)wk, (uint4*)wv, dev_status);
   return cudaGetLastError();
 }

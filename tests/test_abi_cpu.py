@@ -33,7 +33,8 @@ def test_every_declared_function_is_exported(lib):
 
 def test_status_strings(lib):
     assert lib.rf_status_string(0) == b"ok"
-    for code in range(1, 7):
+    assert lib.rf_bounds_checked() == 0
+    for code in range(1, 8):
         assert lib.rf_status_string(code) not in (b"ok", b"unknown status")
     assert lib.rf_status_string(99) == b"unknown status"
 

@@ -29,9 +29,13 @@ from paper_2505_21036_b200 import synth  # noqa: E402
 METRIC = "dense_equiv_tflops_sparse_attn"
 UNIT = "TFLOP/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one rf_attn_kernel launch, from single-pass ncu captures
-# (profiles/rf_attn_kernel_hunyuan720p_dram_bytes.md); None where no capture exists.
+# dram__bytes_read.sum + dram__bytes_write.sum of one rf_attn_kernel launch, from single-pass ncu captures; None
+# where no capture exists.  The figure is a recorded measurement, not taken in this run: TRAFFIC_SOURCE names the
+# summary it comes from and the state of the kernel source it was captured on; re-capture when rf_attn.cu changes.
 ATTN_DRAM_BYTES = {"hunyuan720p": 4.69e9, "sweep_33x3600": 4.69e9, "sweep_16x2040": 0.734e9}
+TRAFFIC_SOURCE = {"file": "profiles/rf_attn_kernel_hunyuan720p_dram_bytes.md",
+                  "captured_on": "rf_attn.cu as of commit 2bbb852 (the kernel body has not changed since)"}
+NOMINAL_BF16_TFLOPS = 2250.0     # NVIDIA's dense bf16 figure for one B200 (the 4.5 PFLOP/s quoted per GPU is with 2:4 sparsity)
 
 
 def peaks():
@@ -305,6 +309,7 @@ def run_cuda(args, wl):
             "breakdown_ms_median": {n: float(np.median(x)) for n, x in stages.items()},
             "breakdown_ms_min": {n: float(np.min(x)) for n, x in stages.items()},
             "arm_overhead_pct": 100.0 * arm_ms / sparse_ms,
+            "arm_plus_mask_overhead_pct": 100.0 * (arm_ms + mask_ms) / sparse_ms,
             "head_classes": {"spatial": int((cls == 0).sum()), "temporal": int((cls == 1).sum()),
                              "textural": int((cls == 2).sum())},
             "recall_mean_by_class": {name: [float(x) for x in rec[cls == c].mean(axis=0)] if (cls == c).any() else None
@@ -317,7 +322,10 @@ def run_cuda(args, wl):
                          "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"], "traffic": ATTN_DRAM_BYTES.get(wl.name),
                          "traffic_unit": "bytes per launch (ncu, dram read + write)",
                          "algorithmic_bytes_per_launch": 4 * wl.B * wl.H * wl.N * wl.D * 2,
+                         "traffic_source": TRAFFIC_SOURCE if ATTN_DRAM_BYTES.get(wl.name) else None,
                          "peak_kind": f"bf16 sustained, of {pk['source']}", "frac_of_burst": achieved / pk["bf16_burst"],
+                         "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+                         "nominal_peak": f"{NOMINAL_BF16_TFLOPS:.0f} TFLOP/s, NVIDIA's dense bf16 figure for one B200",
                          "algorithmic_flops_per_launch": tile_flops},
         }
         # the small kernels against the HBM roofline (algorithmic bytes / measured time)

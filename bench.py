@@ -248,8 +248,8 @@ def run_cuda(args, wl):
     dense_ms = timed(lambda: api.rf_dense_attn_fwd(shape, q, k, v, o, lse, status), 2) if args.dense else None
 
     # end to end with host buffers (pinned): every step moves Q, K, V to the device and O back inside the timed
-    # region.  The library's host-staged call pipelines groups of heads over a copy-in, a compute and a copy-out
-    # stream; the same entry points run as in the device-resident step, once per group.
+    # region, through one C-ABI call (rf_host_pipeline_run) that takes host pointers.  The library pipelines groups of
+    # heads over a copy-in, a compute and a copy-out stream; the same kernels run as in the device-resident step.
     from paper_2505_21036_b200.layer import HostStagedAttention
     heads = wl.B * wl.H
     groups = args.e2e_groups if args.e2e_groups > 0 else next(g for g in (4, 3, 2, 1) if heads % g == 0)
@@ -302,6 +302,7 @@ def run_cuda(args, wl):
             "e2e": {"value": dist_util.replica_throughput(dflops, e2e_ms, world) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": staged.h2d_bytes, "d2h_bytes_per_step": staged.d2h_bytes,
                     "head_groups": groups, "equals_resident_output": e2e_same, "steps": e2e_n,
+                    "api": "rf_host_pipeline_run: one C-ABI call per step with host pointers; the copies are issued inside the library",
                     "overlap": "head groups inside a step; copy-in of the next step under the kernels of this one"},
             "gpu_launches": args.steps * 5,   # rf_arm_kernel, rf_arm_decide_kernel, rf_build_tiles_kernel, rf_gather_kernel, rf_attn_kernel
             "breakdown_ms": {"arm": arm_ms, "block_mask": mask_ms, "sparse_attn_call": sparse_ms, "reorder": reorder_ms,

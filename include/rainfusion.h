@@ -221,6 +221,34 @@ rf_status rf_sparse_attn_fwd_plus(const rf_shape *shape, const rf_params *params
                                   int32_t *dev_status, void *cuda_stream);
 
 /*
+ * The whole path of Fig. 2a (ARM of Sec. 3.3 -> masks of Sec. 3.2 -> masked attention, Eq. 1-2) for callers whose
+ * Q, K, V and O live in HOST memory.  Heads are independent at every stage (Algorithm 1 outputs one category per
+ * head), so a run is pipelined over `head_groups` groups of heads (head_groups must divide B*H) on three streams of
+ * the pipeline's own: copy-in, compute, copy-out.  Every byte of Q, K, V crosses to the device and every byte of O
+ * comes back in every run; only the waiting overlaps, inside a run and between runs made back to back.
+ *   rf_host_pipeline_staging_bytes  host, pure: device bytes the pipeline needs (staged Q, K, V, O for all heads,
+ *                                   workspace and schedule of one group, classes, status).  0 on bad arguments.
+ *   rf_host_pipeline_create         staging: device memory of at least that size, 256-byte aligned, owned by the caller
+ *                                   and handed to the pipeline until it is destroyed.  Creates streams and events only.
+ *   rf_host_pipeline_run            q/k/v/o_host: host bf16 [B,H,N,D], pinned for the copies to overlap; the inputs
+ *                                   must be complete in host memory when the call is made.  Returns when the work is
+ *                                   enqueued; `wait_stream` (a cudaStream_t, NULL = default stream) is made to wait for
+ *                                   the last output copy.  o_host may be read once that stream has been synchronised.
+ *   rf_host_pipeline_status         device int32 the pipeline's kernels report to (dev_status of the calls above)
+ *   rf_host_pipeline_destroy        waits for the pipeline's streams, then releases streams and events
+ * Errors: RF_ERR_INVALID_ARG (null pointers, head_groups not dividing B*H, misaligned staging), RF_ERR_UNSUPPORTED
+ * (head dimension, block size), RF_ERR_WORKSPACE_TOO_SMALL (staging), RF_ERR_CUDA.
+ */
+typedef struct rf_host_pipeline rf_host_pipeline;
+size_t rf_host_pipeline_staging_bytes(const rf_shape *shape, const rf_params *params, int32_t head_groups);
+rf_status rf_host_pipeline_create(const rf_shape *shape, const rf_params *params, int32_t head_groups, void *staging,
+                                  size_t staging_bytes, rf_host_pipeline **out);
+rf_status rf_host_pipeline_run(rf_host_pipeline *p, const void *q_host, const void *k_host, const void *v_host,
+                               void *o_host, void *wait_stream);
+int32_t *rf_host_pipeline_status(rf_host_pipeline *p);
+void rf_host_pipeline_destroy(rf_host_pipeline *p);
+
+/*
  * rf_arm_classify for callers that cannot provide a workspace.  (The paper has no counterpart: this is
  * a packaging variant of rf_arm_classify, same kernels, same results.)
  *

@@ -22,7 +22,8 @@ _lib = None
 EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm_classify",
            "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
            "rf_arm_classify_noalloc", "rf_selftest_wait_timeout", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus",
-           "rf_sparse_attn_reordered", "rf_selftest_arm_abandoned", "rf_bounds_checked"]
+           "rf_sparse_attn_reordered", "rf_selftest_arm_abandoned", "rf_bounds_checked", "rf_host_pipeline_staging_bytes",
+           "rf_host_pipeline_create", "rf_host_pipeline_run", "rf_host_pipeline_status", "rf_host_pipeline_destroy"]
 
 
 class rf_shape(C.Structure):
@@ -58,6 +59,16 @@ def load():
         raise RainFusionError(f"{_LIB_PATH} is missing: build it with `python -m paper_2505_21036_b200.build`")
     lib = C.CDLL(_LIB_PATH)
     P, V, I, Z = C.POINTER, C.c_void_p, C.c_int, C.c_size_t
+    lib.rf_host_pipeline_staging_bytes.restype = Z
+    lib.rf_host_pipeline_staging_bytes.argtypes = [P(rf_shape), P(rf_params), C.c_int32]
+    lib.rf_host_pipeline_create.restype = I
+    lib.rf_host_pipeline_create.argtypes = [P(rf_shape), P(rf_params), C.c_int32, V, Z, P(V)]
+    lib.rf_host_pipeline_run.restype = I
+    lib.rf_host_pipeline_run.argtypes = [V, V, V, V, V, V]
+    lib.rf_host_pipeline_status.restype = V
+    lib.rf_host_pipeline_status.argtypes = [V]
+    lib.rf_host_pipeline_destroy.restype = None
+    lib.rf_host_pipeline_destroy.argtypes = [V]
     lib.rf_bounds_checked.restype = C.c_int32
     lib.rf_bounds_checked.argtypes = []
     lib.rf_status_string.restype = C.c_char_p
@@ -225,6 +236,46 @@ def rf_selftest_arm_abandoned(shape, params, q, k, head_class, ws, dev_status):
     _check(load().rf_selftest_arm_abandoned(C.byref(shape), C.byref(params), q.data_ptr(), k.data_ptr(),
                                             head_class.data_ptr(), ws.data_ptr(), ws.numel(), _ptr(dev_status), _stream()),
            "rf_selftest_arm_abandoned")
+
+
+class HostPipeline:
+    """rf_host_pipeline_*: the whole path with Q, K, V, O in (pinned) host memory, pipelined over groups of heads.
+    torch supplies the staging block; everything else happens behind the C ABI."""
+
+    def __init__(self, shape: rf_shape, params: rf_params, device, head_groups: int):
+        import torch
+        lib = load()
+        n = lib.rf_host_pipeline_staging_bytes(C.byref(shape), C.byref(params), head_groups)
+        if n == 0:
+            raise RainFusionError("rf_host_pipeline_staging_bytes: invalid shape, parameters or head_groups")
+        self.staging = torch.empty(n, dtype=torch.uint8, device=device)
+        h = C.c_void_p()
+        _check(lib.rf_host_pipeline_create(C.byref(shape), C.byref(params), head_groups, self.staging.data_ptr(), n,
+                                           C.byref(h)), "rf_host_pipeline_create")
+        self._h = h
+        self._status_ptr = lib.rf_host_pipeline_status(h)
+
+    def run(self, qh, kh, vh, oh):
+        _check(load().rf_host_pipeline_run(self._h, qh.data_ptr(), kh.data_ptr(), vh.data_ptr(), oh.data_ptr(), _stream()),
+               "rf_host_pipeline_run")
+
+    def status(self) -> int:
+        """The device status word, read back (synchronises)."""
+        import torch
+        torch.cuda.synchronize()
+        off = self._status_ptr - self.staging.data_ptr()
+        return int(self.staging[off:off + 4].view(torch.int32).item())
+
+    def close(self):
+        if self._h is not None:
+            load().rf_host_pipeline_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def rf_reorder_tokens(shape, params, q, k, v, head_class, ws):

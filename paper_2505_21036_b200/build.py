@@ -14,7 +14,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "librainfusion.so")
 LIB_CHECKED = os.path.join(PKG, "librainfusion_checked.so")
-SOURCES = ["rf_api.cu", "rf_mask.cu", "rf_arm.cu", "rf_attn.cu"]
+SOURCES = ["rf_api.cu", "rf_mask.cu", "rf_arm.cu", "rf_attn.cu", "rf_host.cu"]
 HEADERS = ["rf_common.cuh", "rf_sm100.cuh", "rf_attn_common.cuh", os.path.join("..", "..", "include", "rainfusion.h")]
 
 

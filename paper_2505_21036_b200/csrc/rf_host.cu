@@ -1,0 +1,190 @@
+// The whole path for callers whose Q, K, V and O live in host memory, behind the C ABI.
+//
+// Heads are independent at every stage (Algorithm 1 classifies per head; the masks of Sec. 3.2 and the attention of
+// Eq. 1-2 are per head), so a call is pipelined over groups of heads on three streams: while one group's
+// ARM -> tile schedule -> masked attention runs, the next group's inputs arrive from the host and the previous
+// group's output leaves.  Every byte of Q, K, V still crosses to the device and every byte of O comes back in every
+// call; only the waiting overlaps.  Calls made back to back overlap as well: a group's staging buffers are refilled
+// for the next call as soon as this call's kernels have read them.
+// The pipeline object holds streams and events only; device memory comes from the caller in one block.
+#include <new>
+#include <vector>
+
+#include "rf_common.cuh"
+
+struct rf_host_pipeline {
+  rf_shape shape, gshape;       // whole call / one group of heads
+  rf_params params;
+  int groups, heads_per_group;
+  size_t head_elems;            // N * D
+  __nv_bfloat16 *q, *k, *v, *o; // staging, [B*H, N, D]
+  uint8_t* ws;                  // workspace of one group (groups run one after the other on the compute stream)
+  size_t ws_bytes;
+  rf_schedule sched;            // schedule arrays of one group
+  int32_t* head_class;          // [groups, heads_per_group]
+  int32_t* status;
+  cudaStream_t s_in, s_run, s_out;
+  std::vector<cudaEvent_t> landed, run_done, out_done;
+  cudaEvent_t all_done;
+  bool ran;
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+  size_t tensor, ws, count, kv_tile, kv_len, head_class, status, total;
+};
+
+bool layout_of(const rf_shape* shape, const rf_params* params, int groups, rf_shape* gshape, Layout* L, int32_t* nQ, int32_t* nK) {
+  if (shape == nullptr || params == nullptr || groups < 1) return false;
+  const long long heads = (long long)shape->B * shape->H;
+  if (heads < 1 || heads % groups != 0) return false;
+  *gshape = *shape;
+  gshape->B = 1;
+  gshape->H = (int32_t)(heads / groups);
+  if (rf_schedule_dims(gshape, params, nQ, nK) != RF_OK) return false;
+  const size_t ws = rf_workspace_bytes(gshape, params);
+  if (ws == 0) return false;
+  const size_t N = (size_t)shape->T * shape->frame_h * shape->frame_w + shape->L_text;
+  L->tensor = align_up((size_t)heads * N * shape->D * sizeof(__nv_bfloat16));
+  L->ws = align_up(ws);
+  L->count = align_up((size_t)gshape->H * *nQ * sizeof(int32_t));
+  L->kv_tile = align_up((size_t)gshape->H * *nQ * *nK * sizeof(int32_t));
+  L->kv_len = align_up((size_t)gshape->H * sizeof(int32_t));
+  L->head_class = align_up((size_t)heads * sizeof(int32_t));
+  L->status = kAlign;
+  L->total = 4 * L->tensor + L->ws + L->count + L->kv_tile + L->kv_len + L->head_class + L->status;
+  return true;
+}
+
+void destroy(rf_host_pipeline* p) {
+  if (p == nullptr) return;
+  for (auto* vec : {&p->landed, &p->run_done, &p->out_done})
+    for (cudaEvent_t e : *vec)
+      if (e) cudaEventDestroy(e);
+  if (p->all_done) cudaEventDestroy(p->all_done);
+  if (p->s_in) cudaStreamDestroy(p->s_in);
+  if (p->s_run) cudaStreamDestroy(p->s_run);
+  if (p->s_out) cudaStreamDestroy(p->s_out);
+  delete p;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rf_host_pipeline_staging_bytes(const rf_shape* shape, const rf_params* params, int32_t head_groups) {
+  rf_shape gs;
+  Layout L;
+  int32_t nQ, nK;
+  return layout_of(shape, params, head_groups, &gs, &L, &nQ, &nK) ? L.total : 0;
+}
+
+rf_status rf_host_pipeline_create(const rf_shape* shape, const rf_params* params, int32_t head_groups, void* staging,
+                                  size_t staging_bytes, rf_host_pipeline** out) {
+  if (out == nullptr) return RF_ERR_INVALID_ARG;
+  *out = nullptr;
+  rf_shape gs;
+  Layout L;
+  int32_t nQ, nK;
+  if (!layout_of(shape, params, head_groups, &gs, &L, &nQ, &nK)) return RF_ERR_INVALID_ARG;
+  if (shape->D != 64 && shape->D != 96 && shape->D != 128) return RF_ERR_UNSUPPORTED;
+  if (params->block_m != 128 || params->block_n != 128) return RF_ERR_UNSUPPORTED;
+  if (staging == nullptr || (reinterpret_cast<uintptr_t>(staging) & (kAlign - 1)) != 0) return RF_ERR_INVALID_ARG;
+  if (staging_bytes < L.total) return RF_ERR_WORKSPACE_TOO_SMALL;
+  rf_host_pipeline* p = new (std::nothrow) rf_host_pipeline();
+  if (p == nullptr) return RF_ERR_CUDA;
+  p->shape = *shape;
+  p->gshape = gs;
+  p->params = *params;
+  p->groups = head_groups;
+  p->heads_per_group = gs.H;
+  p->head_elems = ((size_t)shape->T * shape->frame_h * shape->frame_w + shape->L_text) * shape->D;
+  uint8_t* b = static_cast<uint8_t*>(staging);
+  p->q = reinterpret_cast<__nv_bfloat16*>(b); b += L.tensor;
+  p->k = reinterpret_cast<__nv_bfloat16*>(b); b += L.tensor;
+  p->v = reinterpret_cast<__nv_bfloat16*>(b); b += L.tensor;
+  p->o = reinterpret_cast<__nv_bfloat16*>(b); b += L.tensor;
+  p->ws = b; p->ws_bytes = L.ws; b += L.ws;
+  p->sched.count = reinterpret_cast<int32_t*>(b); b += L.count;
+  p->sched.kv_tile = reinterpret_cast<int32_t*>(b); b += L.kv_tile;
+  p->sched.kv_len = reinterpret_cast<int32_t*>(b); b += L.kv_len;
+  p->sched.bitmap = nullptr;
+  p->sched.nQ = nQ;
+  p->sched.nKmax = nK;
+  p->head_class = reinterpret_cast<int32_t*>(b); b += L.head_class;
+  p->status = reinterpret_cast<int32_t*>(b);
+  p->s_in = p->s_run = p->s_out = nullptr;
+  p->all_done = nullptr;
+  p->ran = false;
+  bool ok = cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&p->s_run, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p->all_done, cudaEventDisableTiming) == cudaSuccess;
+  for (auto* vec : {&p->landed, &p->run_done, &p->out_done}) {
+    vec->assign(head_groups, nullptr);
+    for (int g = 0; ok && g < head_groups; ++g) ok = cudaEventCreateWithFlags(&(*vec)[g], cudaEventDisableTiming) == cudaSuccess;
+  }
+  ok = ok && cudaMemsetAsync(p->status, 0, sizeof(int32_t), p->s_run) == cudaSuccess &&
+       cudaStreamSynchronize(p->s_run) == cudaSuccess;
+  if (!ok) {
+    destroy(p);
+    return RF_ERR_CUDA;
+  }
+  *out = p;
+  return RF_OK;
+}
+
+void rf_host_pipeline_destroy(rf_host_pipeline* p) {
+  if (p == nullptr) return;
+  cudaStreamSynchronize(p->s_in);
+  cudaStreamSynchronize(p->s_run);
+  cudaStreamSynchronize(p->s_out);
+  destroy(p);
+}
+
+int32_t* rf_host_pipeline_status(rf_host_pipeline* p) { return p ? p->status : nullptr; }
+
+rf_status rf_host_pipeline_run(rf_host_pipeline* p, const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                               void* wait_stream) {
+  if (p == nullptr || q_host == nullptr || k_host == nullptr || v_host == nullptr || o_host == nullptr) return RF_ERR_INVALID_ARG;
+  const size_t gelems = (size_t)p->heads_per_group * p->head_elems, gbytes = gelems * sizeof(__nv_bfloat16);
+  auto at = [&](const void* base, int g) { return static_cast<const uint8_t*>(base) + (size_t)g * gbytes; };
+#define RF_TRY(call) do { if ((call) != cudaSuccess) return RF_ERR_CUDA; } while (0)
+  for (int g = 0; g < p->groups; ++g) {
+    // the previous call's kernels have read this group's staged inputs
+    if (p->ran) RF_TRY(cudaStreamWaitEvent(p->s_in, p->run_done[g], 0));
+    RF_TRY(cudaMemcpyAsync(p->q + g * gelems, at(q_host, g), gbytes, cudaMemcpyHostToDevice, p->s_in));
+    RF_TRY(cudaMemcpyAsync(p->k + g * gelems, at(k_host, g), gbytes, cudaMemcpyHostToDevice, p->s_in));
+    RF_TRY(cudaMemcpyAsync(p->v + g * gelems, at(v_host, g), gbytes, cudaMemcpyHostToDevice, p->s_in));
+    RF_TRY(cudaEventRecord(p->landed[g], p->s_in));
+  }
+  for (int g = 0; g < p->groups; ++g) {
+    RF_TRY(cudaStreamWaitEvent(p->s_run, p->landed[g], 0));
+    // the previous call's output of this group has left the staging buffer
+    if (p->ran) RF_TRY(cudaStreamWaitEvent(p->s_run, p->out_done[g], 0));
+    int32_t* hc = p->head_class + (size_t)g * p->heads_per_group;
+    const __nv_bfloat16 *q = p->q + g * gelems, *k = p->k + g * gelems, *v = p->v + g * gelems;
+    rf_status st = rf_arm_classify(&p->gshape, &p->params, q, k, hc, nullptr, p->ws, p->ws_bytes, p->status, p->s_run);
+    if (st == RF_OK) st = rf_build_block_mask(&p->gshape, &p->params, hc, &p->sched, p->status, p->s_run);
+    if (st == RF_OK)
+      st = rf_sparse_attn_fwd(&p->gshape, &p->params, q, k, v, hc, &p->sched, p->o + g * gelems, nullptr, p->ws, p->ws_bytes,
+                              p->status, p->s_run);
+    if (st != RF_OK) return st;
+    RF_TRY(cudaEventRecord(p->run_done[g], p->s_run));
+    RF_TRY(cudaStreamWaitEvent(p->s_out, p->run_done[g], 0));
+    RF_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(o_host) + (size_t)g * gbytes, p->o + g * gelems, gbytes, cudaMemcpyDeviceToHost,
+                           p->s_out));
+    RF_TRY(cudaEventRecord(p->out_done[g], p->s_out));
+  }
+  p->ran = true;
+  RF_TRY(cudaEventRecord(p->all_done, p->s_out));
+  RF_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(wait_stream), p->all_done, 0));
+#undef RF_TRY
+  return RF_OK;
+}
+
+}  // extern "C"

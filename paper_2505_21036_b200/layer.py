@@ -95,73 +95,36 @@ class RainFusionAttention:
 
 
 class HostStagedAttention:
-    """The whole path for callers whose Q, K, V and O live in (pinned) host memory.
-
-    Heads are independent at every stage (Algorithm 1 classifies per head; masks and attention are per head), so
-    the call is pipelined over groups of heads: while one group's ARM -> schedule -> masked attention runs, the next
-    group's inputs arrive on a copy stream and the previous group's output leaves on another.  Per step every byte
-    of Q, K, V still crosses to the device and every byte of O comes back; only the waiting is overlapped.
-    """
+    """The whole path for callers whose Q, K, V and O live in (pinned) host memory: a thin wrapper over the
+    library's rf_host_pipeline_* calls, which pipeline groups of heads over a copy-in, a compute and a copy-out
+    stream (heads are independent at every stage: Algorithm 1 classifies per head; masks and attention are per
+    head).  Per call every byte of Q, K, V still crosses to the device and every byte of O comes back; only the
+    waiting is overlapped, inside a call and between calls made back to back."""
 
     def __init__(self, shape: api.rf_shape, params: api.rf_params, device, groups: int = 4):
-        import torch
         heads = shape.B * shape.H
         if groups < 1 or heads % groups != 0:
             raise ValueError("groups must divide B*H")
         self.shape, self.params, self.device, self.groups = shape, params, device, groups
-        self.hg = heads // groups
-        self.gshape = api.rf_shape(1, self.hg, shape.D, shape.T, shape.frame_h, shape.frame_w, shape.L_text)
         self.N = shape.T * shape.frame_h * shape.frame_w + shape.L_text
-        dims = (heads, self.N, shape.D)
-        self.q, self.k, self.v, self.o = (torch.empty(dims, dtype=torch.bfloat16, device=device) for _ in range(4))
-        self.ws = api.alloc_workspace(self.gshape, params, device)
-        self.sched = api.Schedule(self.gshape, params, device)
-        self.head_class = torch.zeros((groups, self.hg), dtype=torch.int32, device=device)
-        self.status = torch.zeros(1, dtype=torch.int32, device=device)
-        self.s_in, self.s_run, self.s_out = (torch.cuda.Stream(device=device) for _ in range(3))
-        self._run_done, self._out_done = [], []      # per group, from the previous call
+        self.pipe = api.HostPipeline(shape, params, device, groups)
         self.h2d_bytes = 3 * heads * self.N * shape.D * 2
         self.d2h_bytes = heads * self.N * shape.D * 2
 
     def __call__(self, qh, kh, vh, oh):
         """qh, kh, vh, oh: pinned host bf16 tensors of [B, H, N, D]; the inputs must be complete in host memory
-        when the call is made.  Returns when the work is enqueued; the current stream waits for the output copy.
-        Calls made back to back overlap: a group's staging buffers are refilled for the next call as soon as
-        this call's kernels are done with them, while later groups still compute."""
-        import torch
-        cur = torch.cuda.current_stream()
-        hq, hk, hv, ho = (t.view(self.groups, self.hg, self.N, self.shape.D) for t in (qh, kh, vh, oh))
-        dq, dk, dv, do = (t.view(self.groups, self.hg, self.N, self.shape.D) for t in (self.q, self.k, self.v, self.o))
-        prev_run, prev_out = self._run_done, self._out_done
-        landed, run_done, out_done = [], [], []
-        with torch.cuda.stream(self.s_in):
-            for g in range(self.groups):
-                if prev_run:
-                    self.s_in.wait_event(prev_run[g])      # the previous call's kernels have read this group's inputs
-                dq[g].copy_(hq[g], non_blocking=True)
-                dk[g].copy_(hk[g], non_blocking=True)
-                dv[g].copy_(hv[g], non_blocking=True)
-                ev = torch.cuda.Event()
-                ev.record()
-                landed.append(ev)
-        for g in range(self.groups):
-            with torch.cuda.stream(self.s_run):
-                self.s_run.wait_event(landed[g])
-                if prev_out:
-                    self.s_run.wait_event(prev_out[g])     # the previous call's output of this group has left
-                hc = self.head_class[g:g + 1]
-                api.rf_arm_classify(self.gshape, self.params, dq[g], dk[g], hc, None, self.ws, self.status)
-                api.rf_build_block_mask(self.gshape, self.params, hc, self.sched, self.status)
-                api.rf_sparse_attn_fwd(self.gshape, self.params, dq[g], dk[g], dv[g], hc, self.sched, do[g], None, self.ws,
-                                       self.status)
-                done = torch.cuda.Event()
-                done.record()
-                run_done.append(done)
-            with torch.cuda.stream(self.s_out):
-                self.s_out.wait_event(done)
-                ho[g].copy_(do[g], non_blocking=True)
-                ev = torch.cuda.Event()
-                ev.record()
-                out_done.append(ev)
-        self._run_done, self._out_done = run_done, out_done
-        cur.wait_stream(self.s_out)
+        when the call is made.  Returns when the work is enqueued; the current stream waits for the output copy."""
+        for t in (qh, kh, vh, oh):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("host-staged call takes contiguous host tensors")
+        self.pipe.run(qh, kh, vh, oh)
+
+    @property
+    def status(self):
+        """Object with .item(): the pipeline's device status word."""
+        pipe = self.pipe
+
+        class _S:
+            def item(self_inner):
+                return pipe.status()
+        return _S()

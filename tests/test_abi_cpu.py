@@ -103,6 +103,28 @@ def test_oversized_windows_and_strides_are_accepted_and_bounded(lib):
     assert time.time() - t0 < 0.5
 
 
+def test_host_pipeline_arguments_are_checked_before_cuda(lib):
+    wl = synth.WORKLOADS["tiny"]                       # 3 heads
+    s, p = api.shape_of(wl), api.params_of(wl)
+    full = lib.rf_host_pipeline_staging_bytes(C.byref(s), C.byref(p), 1)
+    per3 = lib.rf_host_pipeline_staging_bytes(C.byref(s), C.byref(p), 3)
+    tensor = -(-(wl.B * wl.H * wl.N * wl.D * 2) // 256) * 256
+    assert full >= 4 * tensor + api.rf_workspace_bytes(s, p) and 4 * tensor < per3 < full   # one group's workspace and schedule
+    assert lib.rf_host_pipeline_staging_bytes(C.byref(s), C.byref(p), 2) == 0           # 2 does not divide 3 heads
+    assert lib.rf_host_pipeline_staging_bytes(C.byref(s), C.byref(p), 0) == 0
+    h = C.c_void_p()
+    assert lib.rf_host_pipeline_create(C.byref(s), C.byref(p), 2, 256, 1 << 40, C.byref(h)) == 1
+    assert lib.rf_host_pipeline_create(C.byref(s), C.byref(p), 3, 264, 1 << 40, C.byref(h)) == 1   # misaligned staging
+    assert lib.rf_host_pipeline_create(C.byref(s), C.byref(p), 3, 256, per3 - 1, C.byref(h)) == 3  # staging too small
+    assert lib.rf_host_pipeline_create(C.byref(s), C.byref(p), 3, None, per3, C.byref(h)) == 1
+    p64 = api.params_of(wl, 64, 64)
+    assert lib.rf_host_pipeline_create(C.byref(s), C.byref(p64), 3, 256, 1 << 40, C.byref(h)) == 2  # attention needs 128 x 128 tiles
+    assert h.value is None
+    assert lib.rf_host_pipeline_run(None, 256, 256, 256, 256, None) == 1
+    assert lib.rf_host_pipeline_status(None) is None
+    lib.rf_host_pipeline_destroy(None)                 # a no-op
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(api, "_lib", None)
     monkeypatch.setattr(api, "_LIB_PATH", str(tmp_path / "nope.so"))

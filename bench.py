@@ -32,9 +32,9 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one rf_attn_kernel launch, from single-pass ncu captures; None
 # where no capture exists.  The figure is a recorded measurement, not taken in this run: TRAFFIC_SOURCE names the
 # summary it comes from and the state of the kernel source it was captured on; re-capture when rf_attn.cu changes.
-ATTN_DRAM_BYTES = {"hunyuan720p": 4.69e9, "sweep_33x3600": 4.69e9, "sweep_16x2040": 0.734e9}
+ATTN_DRAM_BYTES = {"hunyuan720p": 4.67e9, "sweep_33x3600": 4.67e9, "sweep_16x2040": 0.734e9}
 TRAFFIC_SOURCE = {"file": "profiles/rf_attn_kernel_hunyuan720p_dram_bytes.md",
-                  "captured_on": "rf_attn.cu as of commit 2bbb852 (the kernel body has not changed since)"}
+                  "captured_on": "the kernel as of the commit that last touched profiles/ (its body is that of commit 2bbb852)"}
 NOMINAL_BF16_TFLOPS = 2250.0     # NVIDIA's dense bf16 figure for one B200 (the 4.5 PFLOP/s quoted per GPU is with 2:4 sparsity)
 
 

@@ -15,7 +15,8 @@ fp64 exactly.
 Readings taken where the paper is silent (each also listed in the design notes):
   * tokens: frame-major, row-major inside a frame, text tokens appended last;
   * Spatial head keeps |frame(i) - frame(j)| <= w_f (Eq. 3: the significant frames
-    of frame f are its neighbours); Temporal head keeps |pos(i) - pos(j)| <= w_s with
+    of frame f are its neighbours); as an option (Sec. 3.2 speaks of adjacent OR key frames) the
+    first frame counts as a key frame that every query keeps as well; Temporal head keeps |pos(i) - pos(j)| <= w_s with
     pos the flattened in-frame index (Sec. 3.2 describes Temporal heads as local inside one
     frame's sub-sequence and periodic across frames); text rows and text columns are always kept for both;
   * Textural head keeps key/value token (y, x) of every frame iff y mod tau == x mod tau
@@ -69,6 +70,7 @@ class PatternParams:
     frame_window: int      # w_f
     spatial_window: int    # w_s
     textural_stride: int   # tau
+    keep_first_frame: bool = False   # Spatial heads also keep every key of frame 0 (a "key frame", Sec. 3.2)
 
 
 def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
@@ -107,6 +109,8 @@ def keep_mask(pattern: int, rows: np.ndarray, cols: np.ndarray, g: Geometry, pp:
         return np.ones((i.shape[0], j.shape[1]), dtype=bool)
     if pattern == SPATIAL:
         near = np.abs(frame_of(i, g) - frame_of(j, g)) <= pp.frame_window
+        if pp.keep_first_frame:
+            near = near | (frame_of(j, g) == 0)
         return i_text | j_text | near
     if pattern == TEMPORAL:
         near = np.abs(pos_of(i, g) - pos_of(j, g)) <= pp.spatial_window
@@ -233,7 +237,7 @@ def decide_plus(R_temporal: Sequence[float], R_spatial: Sequence[float], alpha: 
 
 
 def arm_head_plus(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, bandwidths: Sequence[float], tau: int,
-                  sample_mode: int, omega: int, alpha: float, two_mask: bool = False):
+                  sample_mode: int, omega: int, alpha: float, two_mask: bool = False, keep_first_frame: bool = False):
     """ARM with dynamic bandwidth for one head: every candidate bandwidth's Temporal and Spatial recall on
     the same approximate scores, then decide_plus.  Returns (class, index, window, R_t list, R_s list),
     window = w_s of the chosen bandwidth for Temporal, w_f for Spatial, -1 for Textural."""
@@ -247,7 +251,7 @@ def arm_head_plus(q_bits: np.ndarray, k_bits: np.ndarray, g: Geometry, bandwidth
     R_t, R_s = [], []
     for b in bandwidths:
         wf, ws = windows_of(b, g)
-        pp = PatternParams(wf, ws, tau)
+        pp = PatternParams(wf, ws, tau, keep_first_frame)
         R_t.append(recall(P_t, keep_mask(TEMPORAL, I_t, I_t, g, pp)))
         R_s.append(recall(P_glb, keep_mask(SPATIAL, I_glb, I_glb, g, pp)))
     cls, idx = decide_plus(R_t, R_s, alpha, two_mask)

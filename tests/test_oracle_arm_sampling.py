@@ -174,3 +174,27 @@ def test_spatial_recall_never_comes_from_the_first_frame():
 ])
 def test_bandwidth_to_window_takes_the_floor(b, T, fh, fw, expect):
     assert orc.windows_of(b, Geometry(T, fh, fw, 0)) == expect
+
+
+def test_spatial_recall_with_the_first_frame_as_key_frame(qk):
+    """Option of Sec. 3.2's "adjacent or key frames": the sampled Spatial mask also keeps the sampled keys of frame 0;
+    the Temporal recall does not change."""
+    q, k = qk
+    strided = list(range(0, G.Nv, OMEGA))
+    n = len(strided)
+    kept = np.zeros((n, n), dtype=bool)
+    for a in range(n):
+        for b in range(n):
+            kept[a, b] = abs(strided[a] // G.S - strided[b] // G.S) <= PP.frame_window or strided[b] // G.S == 0
+    expect = recall_by_library(q, k, strided, kept)
+    pp_on = PatternParams(PP.frame_window, PP.spatial_window, PP.textural_stride, True)
+    _, (rt_on, rs_on, _), _ = orc.arm_head(q, k, G, pp_on, orc.SAMPLE_ALG1, OMEGA, 0.9)
+    _, (rt_off, rs_off, _), _ = orc.arm_head(q, k, G, PP, orc.SAMPLE_ALG1, OMEGA, 0.9)
+    assert rs_on == pytest.approx(expect, abs=1e-12) and rs_on > rs_off + 1e-3 and rt_on == rt_off
+    _, _, _, Rt, Rs = orc.arm_head_plus(q, k, G, [0.2, 0.45], 2, orc.SAMPLE_ALG1, OMEGA, 0.9, keep_first_frame=True)
+    kept2 = np.zeros((n, n), dtype=bool)
+    for a in range(n):
+        for b in range(n):
+            kept2[a, b] = abs(strided[a] // G.S - strided[b] // G.S) <= 2 or strided[b] // G.S == 0     # floor(0.45 * 5) = 2
+    assert Rs[0] == pytest.approx(expect, abs=1e-12)                                                  # floor(0.2 * 5) = 1 = PP's window
+    assert Rs[1] == pytest.approx(recall_by_library(q, k, strided, kept2), abs=1e-12)

@@ -268,3 +268,54 @@ def test_permutation_makes_temporal_mask_banded():
     for r in range(g.Nv):
         nz = np.flatnonzero(M[r])
         assert nz[-1] - nz[0] + 1 == len(nz)
+
+
+# ---------------------------------------------------------------- Spatial head with the first frame as a key frame
+
+def test_key_first_frame_mask_by_enumeration():
+    """Sec. 3.2 lets a Spatial head attend adjacent OR key frames; with the option on, every query also keeps the keys
+    of frame 0.  Nested loops over the definition, all patterns (only Spatial may change)."""
+    g = Geometry(5, 2, 3, 2)
+    idx = np.arange(g.N)
+    for wf in (0, 1, 2):
+        on, off = PatternParams(wf, 1, 2, True), PatternParams(wf, 1, 2, False)
+        M = orc.keep_mask(SPATIAL, idx, idx, g, on)
+        for i in range(g.N):
+            for j in range(g.N):
+                if i >= g.Nv or j >= g.Nv:
+                    want = True
+                else:
+                    want = abs(i // g.S - j // g.S) <= wf or j // g.S == 0
+                assert M[i, j] == want, (wf, i, j)
+        for pattern in (TEMPORAL, TEXTURAL, DENSE):
+            assert np.array_equal(orc.keep_mask(pattern, idx, idx, g, on), orc.keep_mask(pattern, idx, idx, g, off))
+        # a superset of the plain Spatial mask that differs only in key columns of frame 0
+        P = orc.keep_mask(SPATIAL, idx, idx, g, off)
+        assert (M | P).sum() == M.sum() and np.array_equal(M[:, g.S:], P[:, g.S:])
+
+
+def test_key_first_frame_kept_fraction_closed_form():
+    # frame pairs kept: the band T(2w+1) - w(w+1) plus, in key column 0, the query frames the band does not reach: T - 1 - w
+    for T, w in ((8, 1), (13, 3), (6, 0), (5, 4), (5, 9)):
+        g = Geometry(T, 2, 2, 0)
+        idx = np.arange(g.N)
+        M = orc.keep_mask(SPATIAL, idx, idx, g, PatternParams(w, 0, 2, True))
+        wc = min(w, T - 1)
+        frames = T * (2 * wc + 1) - wc * (wc + 1) + (T - 1 - wc)
+        assert M.sum() == frames * g.S * g.S
+
+
+def test_key_first_frame_tile_lists_follow_the_mask():
+    g = Geometry(6, 4, 8, 5)                     # S = 32: a 16-slot tile never straddles two frames, a 64-slot tile always does
+    pp = PatternParams(1, 3, 2, True)
+    pq = orc.query_order(SPATIAL, g, False)
+    kept = orc.keep_mask(SPATIAL, pq, pq, g, pp)
+    for block in (16, 64):
+        nQ = -(-g.N // block)
+        for a in range(nQ):
+            row = orc.tile_row(SPATIAL, g, pp, False, block, block, a)
+            tiles = [e & ~orc.PARTIAL_BIT for e in row]
+            assert 0 in tiles                      # the first key tile lies in frame 0: every query tile lists it
+            for b in range(nQ):
+                sub = kept[a * block:(a + 1) * block, b * block:(b + 1) * block]
+                assert (b in tiles) == bool(sub.any())

@@ -79,6 +79,9 @@ typedef struct {
   int32_t two_mask;         /* 0: Algorithm 1 as printed (Spatial, Temporal, else Textural).  1: the ablation of
                                Sec. 4.4 / Table 2 with only the Spatial and Temporal masks: a head that reaches alpha
                                with neither takes the one of larger recall (Temporal on equality), never Textural */
+  int32_t spatial_key_first_frame; /* 0: a Spatial head keeps the frames within w_f (Eq. 3).  1: it keeps, in addition,
+                               every key of frame 0 for every query: Sec. 3.2 lets the attended set hold adjacent
+                               or key frames; the first frame is the one key frame offered here */
 } rf_params;
 
 /*

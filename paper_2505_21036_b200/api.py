@@ -34,7 +34,7 @@ class rf_params(C.Structure):
     _fields_ = [("frame_window", C.c_int32), ("spatial_window", C.c_int32), ("textural_stride", C.c_int32),
                 ("sample_mode", C.c_int32), ("sample_stride", C.c_int32), ("alpha", C.c_float),
                 ("block_m", C.c_int32), ("block_n", C.c_int32), ("temporal_permute", C.c_int32),
-                ("two_mask", C.c_int32)]
+                ("two_mask", C.c_int32), ("spatial_key_first_frame", C.c_int32)]
 
 
 class rf_schedule(C.Structure):
@@ -125,9 +125,9 @@ def make_shape(B, H, D, T, frame_h, frame_w, L_text) -> rf_shape:
 
 
 def make_params(frame_window, spatial_window, textural_stride=2, sample_mode=RF_SAMPLE_ALG1, sample_stride=1,
-                alpha=0.9, block_m=128, block_n=128, temporal_permute=1, two_mask=0) -> rf_params:
+                alpha=0.9, block_m=128, block_n=128, temporal_permute=1, two_mask=0, spatial_key_first_frame=0) -> rf_params:
     return rf_params(frame_window, spatial_window, textural_stride, sample_mode, sample_stride, alpha,
-                     block_m, block_n, temporal_permute, two_mask)
+                     block_m, block_n, temporal_permute, two_mask, spatial_key_first_frame)
 
 
 def shape_of(wl) -> rf_shape:
@@ -135,10 +135,10 @@ def shape_of(wl) -> rf_shape:
     return rf_shape(wl.B, wl.H, wl.D, wl.T, wl.frame_h, wl.frame_w, wl.L_text)
 
 
-def params_of(wl, block_m=128, block_n=128, temporal_permute=1, two_mask=0) -> rf_params:
+def params_of(wl, block_m=128, block_n=128, temporal_permute=1, two_mask=0, spatial_key_first_frame=0) -> rf_params:
     """rf_params of a synth.Workload."""
     return rf_params(wl.frame_window, wl.spatial_window, wl.textural_stride, wl.sample_mode, wl.sample_stride,
-                     wl.alpha, block_m, block_n, temporal_permute, two_mask)
+                     wl.alpha, block_m, block_n, temporal_permute, two_mask, spatial_key_first_frame)
 
 
 def rf_schedule_dims(shape: rf_shape, params: rf_params):

@@ -29,6 +29,7 @@ rf_status check_params(const rf_params* p) {
   if (!pow2(p->block_m) || !pow2(p->block_n) || p->block_m < 16 || p->block_n < 16) return RF_ERR_INVALID_ARG;
   if (p->temporal_permute != 0 && p->temporal_permute != 1) return RF_ERR_INVALID_ARG;
   if (p->two_mask != 0 && p->two_mask != 1) return RF_ERR_INVALID_ARG;
+  if (p->spatial_key_first_frame != 0 && p->spatial_key_first_frame != 1) return RF_ERR_INVALID_ARG;
   return RF_OK;
 }
 
@@ -62,11 +63,13 @@ RfGeom make_geom(const rf_shape* s, int wf, int ws, int tau, int bm, int bn, int
   g.nKmax = rf_cdiv(g.N, bn);
   g.permute = permute;
   g.two_mask = 0;
+  g.key_first = 0;
   return g;
 }
 RfGeom make_geom(const rf_shape* s, const rf_params* p) {
   RfGeom g = make_geom(s, p->frame_window, p->spatial_window, p->textural_stride, p->block_m, p->block_n, p->temporal_permute);
   g.two_mask = p->two_mask;
+  g.key_first = p->spatial_key_first_frame;
   return g;
 }
 

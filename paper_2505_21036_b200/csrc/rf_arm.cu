@@ -16,6 +16,8 @@
 // it for all 32 rows of a warp cost nothing extra, tiles an edge crosses use a 128-bit keep word per
 // row.  Only the Temporal mask on the stride sample (RF_SAMPLE_GLOBAL) and the Textural diagnostic
 // need per-key attributes, computed cooperatively per tile.
+// With the first frame as a key frame of Spatial heads (Sec. 3.2: adjacent or key frames) the Spatial masks keep,
+// in addition, the sampled keys of frame 0, a prefix of the stride sample.
 // Per-row recalls go to scratch; a second kernel averages them in a fixed order (deterministic) and
 // takes Algorithm 1's decision.  The n x n score matrix is never written.
 // A bounded wait that runs out is recorded in a flag word at the end of the scratch (cleared at the start of
@@ -268,12 +270,15 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
           if (is_x ? !TEX : (is_t ? !sm.want_t : !sm.want_s)) continue;
           const bool by_table = is_x || (is_t && t_generic);
           int cls = 1;
-          int klo = 0, khi = 0;
+          int klo = 0, khi = 0, pre = 0;
           if (!by_table) {
 #pragma unroll
             for (int i = 0; i < 2 * NB; ++i)
               if (i == k) { klo = lo[i]; khi = hi[i]; }
-            const bool in = klo <= u0 && u1 <= khi, out = u1 <= klo || khi <= u0;
+            // Spatial masks with the first frame as key frame also keep the sampled keys of frame 0: a prefix
+            // [0, pre) of the stride sample, the same for every row
+            pre = (!is_t && g.key_first) ? rf_cdiv(g.S, stride) : 0;
+            const bool in = (klo <= u0 && u1 <= khi) || u1 <= pre, out = (u1 <= klo || khi <= u0) && u0 >= pre;
             cls = __all_sync(0xffffffffu, in) ? 2 : (__all_sync(0xffffffffu, out) ? 0 : 1);
           }
           float add = 0.f;
@@ -283,6 +288,12 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
             uint32_t w[4] = {0, 0, 0, 0};
             if (!by_table) {
               interval_bits(w, u0, klo, khi);
+              if (pre > u0) {
+                uint32_t wp[4];
+                interval_bits(wp, u0, 0, pre);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) w[q4] |= wp[q4];
+              }
             } else {
               if (!table_ready) {
                 // per-key attributes of the tile, four keys per lane, into this warp's table

@@ -30,6 +30,7 @@ __device__ __forceinline__ float ex2(float x) {
 // rare, and a large rarely-run code block costs more in instruction fetch than in arithmetic.
 struct RowMask {
   int lo, hi;        // kept video slots [lo, hi) when !periodic
+  int first_end;     // slots [0, first_end) are kept as well (Spatial with the first frame as key frame), else 0
   int text0;         // first always-kept (text) slot
   int lkv;           // number of key slots
   int p, ws, S, T;   // periodic form: |slot % S - p| <= ws for slots of frames 0..T-1
@@ -56,6 +57,7 @@ struct RowMask {
       for (int f = u0 / S; f <= f1; ++f) add(w, u0, f * S + max(p - ws, 0), f * S + min(p + ws, S - 1) + 1);
     } else {
       add(w, u0, lo, min(hi, text0));
+      add(w, u0, 0, first_end);
     }
     add(w, u0, text0, lkv);
   }
@@ -67,6 +69,7 @@ __device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r
   m.text0 = m.lkv;
   m.lo = 0;
   m.hi = m.lkv;
+  m.first_end = 0;
   m.p = 0; m.ws = g.ws; m.S = g.S; m.T = g.T;
   m.periodic = false;
   if ((cls == RF_SPATIAL || cls == RF_TEMPORAL) && r < g.Nv) {
@@ -75,6 +78,7 @@ __device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r
       const int f = r / g.S;
       m.lo = max(0, f - g.wf) * g.S;
       m.hi = min(g.T, f + g.wf + 1) * g.S;
+      m.first_end = g.key_first ? g.S : 0;
     } else if (g.permute) {
       const int p = r / g.T;
       m.lo = max(0, p - g.ws) * g.T;

@@ -21,6 +21,7 @@ struct RfGeom {
   int BM, BN, nQ, nKmax; // block mask tile and its extents
   int permute;           // Temporal heads in position-major order
   int two_mask;          // ARM decides between Spatial and Temporal only (ablation of Sec. 4.4)
+  int key_first;         // Spatial heads also keep every key of frame 0 (a key frame, Sec. 3.2)
 };
 
 // Device-side error reporting: first error wins, kernels never trap.

@@ -43,6 +43,12 @@ __device__ int tile_flag(const RfGeom& g, int cls, int a, int b) {
         const int ra = r0 / unit, rb = (rv1 - 1) / unit, ca = u0 / unit, cb = (uv1 - 1) / unit;
         vv_any = max(max(ca - rb, ra - cb), 0) <= w;
         vv_all = max(rb - ca, cb - ra) <= w;
+        if (cls == RF_SPATIAL && g.key_first) {
+          // keys of frame 0 are kept for every query: the tile is non-empty if it reaches into frame 0, and all of
+          // it is kept if the window holds for its keys of the other frames (if it has any)
+          vv_any = vv_any || ca == 0;
+          vv_all = cb == 0 || max(rb - max(ca, 1), cb - ra) <= w;
+        }
       } else {
         Iv R[2], C[2];
         const int nr = cyclic_intervals(r0, rv1, g.S, R), nc = cyclic_intervals(u0, uv1, g.S, C);

@@ -53,7 +53,7 @@ def test_schedule_dims_and_workspace_for_every_workload(lib):
 @pytest.mark.parametrize("field,value", [("frame_window", -1), ("spatial_window", -1), ("textural_stride", 0),
                                          ("sample_stride", 0), ("sample_mode", 2), ("alpha", 0.0), ("alpha", 1.5),
                                          ("block_m", 48), ("block_n", 8), ("temporal_permute", 2), ("two_mask", 2),
-                                         ("two_mask", -1)])
+                                         ("two_mask", -1), ("spatial_key_first_frame", 2), ("spatial_key_first_frame", -1)])
 def test_bad_parameters_are_rejected(lib, field, value):
     wl = synth.WORKLOADS["tiny"]
     s, p = api.shape_of(wl), api.params_of(wl)

@@ -454,3 +454,49 @@ def test_row_maximum_growing_in_late_tiles(D):
     gu.check_attention(O[0, 0], lse[0, 0], *ref_d, "staircase sparse/dense-class", strict=False)
     gu.check_attention(O[0, 1], lse[0, 1], *ref_x, "staircase textural", strict=False)
     gu.check_attention(Od[0, 1], lsed[0, 1], *ref_d, "staircase dense entry", strict=False)
+
+
+# ------------------------------------------------------------------ Spatial heads with the first frame as key frame
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_first_frame_as_key_frame(mode):
+    """Sec. 3.2 lets a Spatial head attend adjacent or key frames: with spatial_key_first_frame every query also keeps
+    the keys of frame 0.  ARM's Spatial recall, the tile lists at several tile sizes and the attention output against the
+    oracle; the other patterns must not change."""
+    for kw in (dict(T=6, fh=12, fw=11, L=37, wf=1, ws=20, omega=6), dict(T=9, fh=5, fw=8, L=0, wf=0, ws=3, omega=7),
+               dict(T=4, fh=20, fw=20, L=9, wf=2, ws=50, omega=3)):
+        wl = synth.small_workload("key_first", H=4, D=64, mode=mode, amp=1.5, **kw)
+        g, pp = gu.geom(wl), gu.pparams(wl, True)
+        run = gu.Run(wl, key_first=1)
+        cls_gpu, rec_gpu = run.arm()
+        cls_ref, rec_ref, margin = orc.arm_classify(run.q_bits, run.k_bits, g, pp, wl.sample_mode, wl.sample_stride, wl.alpha)
+        assert np.abs(rec_gpu - rec_ref).max() <= gu.RECALL_ABS, np.abs(rec_gpu - rec_ref).max()
+        decided = margin > gu.TIE_MARGIN
+        assert np.array_equal(cls_gpu[decided], cls_ref[decided])
+        plain = gu.Run(wl)
+        _, rec_plain = plain.arm()
+        assert (rec_gpu[..., 1] >= rec_plain[..., 1] - 1e-6).all() and np.allclose(rec_gpu[..., 0], rec_plain[..., 0], atol=1e-6)
+        classes = [S_, T_, X_, D_]
+        run.force_classes(classes)
+        run.build()
+        O, lse = run.sparse()
+        for h, cls in enumerate(classes):
+            ref = gu.oracle_lists(wl, cls, 128, 1, key_first=True)
+            assert run.lists(0, h) == [ref[a] for a in range(run.sched.nQ)], (kw, cls)
+            Or, lr = orc.masked_attention(run.q_bits[0, h], run.k_bits[0, h], run.v_bits[0, h], cls, g, pp)
+            gu.check_attention(O[0, h], lse[0, h], Or, lr, f"key first frame, class {cls}", strict=False)
+        # dynamic bandwidth: every candidate's Spatial recall carries the key frame too
+        bws = [0.2, 0.5]
+        plus = gu.Run(wl, key_first=1)
+        _, _, rec_plus = plus.arm_plus(bws)
+        for h in range(wl.H):
+            _, _, _, Rt, Rs = orc.arm_head_plus(run.q_bits[0, h], run.k_bits[0, h], g, bws, wl.textural_stride, wl.sample_mode,
+                                                wl.sample_stride, wl.alpha, keep_first_frame=True)
+            assert np.abs(rec_plus[0, h, 0] - np.asarray(Rt)).max() <= gu.RECALL_ABS
+            assert np.abs(rec_plus[0, h, 1] - np.asarray(Rs)).max() <= gu.RECALL_ABS
+        for block in (16, 32, 64):
+            small = gu.Run(wl, block=block, key_first=1)
+            small.force_classes(classes)
+            small.build()
+            ref = gu.oracle_lists(wl, S_, block, 1, key_first=True)
+            assert small.lists(0, 0) == [ref[a] for a in range(small.sched.nQ)], (kw, block)

@@ -18,7 +18,9 @@ Readings taken where the paper is silent (each also listed in the design notes):
     of frame f are its neighbours); as an option (Sec. 3.2 speaks of adjacent OR key frames) the
     first frame counts as a key frame that every query keeps as well; Temporal head keeps |pos(i) - pos(j)| <= w_s with
     pos the flattened in-frame index (Sec. 3.2 describes Temporal heads as local inside one
-    frame's sub-sequence and periodic across frames); text rows and text columns are always kept for both;
+    frame's sub-sequence and periodic across frames); as an option the locality is a 2-D window
+    |y(i) - y(j)| <= w_y and |x(i) - x(j)| <= w_x on the frame's rows and columns, the other way to read
+    "local" for tokens that are image patches; text rows and text columns are always kept for both;
   * Textural head keeps key/value token (y, x) of every frame iff y mod tau == x mod tau
     (Eq. 4), plus all text keys, for every query (Eq. 5: all-zero mask on K_C, V_C);
   * recall (Eq. 6) is the share of a row's unmasked softmax mass that falls on kept
@@ -71,6 +73,8 @@ class PatternParams:
     spatial_window: int    # w_s
     textural_stride: int   # tau
     keep_first_frame: bool = False   # Spatial heads also keep every key of frame 0 (a "key frame", Sec. 3.2)
+    temporal_window_2d: Optional[Tuple[int, int]] = None   # (w_y, w_x): Temporal heads keep |y(i)-y(j)| <= w_y and
+                                                           # |x(i)-x(j)| <= w_x instead of the 1-D band on the flattened index
 
 
 def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
@@ -113,7 +117,12 @@ def keep_mask(pattern: int, rows: np.ndarray, cols: np.ndarray, g: Geometry, pp:
             near = near | (frame_of(j, g) == 0)
         return i_text | j_text | near
     if pattern == TEMPORAL:
-        near = np.abs(pos_of(i, g) - pos_of(j, g)) <= pp.spatial_window
+        if pp.temporal_window_2d is not None:
+            wy, wx = pp.temporal_window_2d
+            pi, pj = pos_of(i, g), pos_of(j, g)
+            near = (np.abs(pi // g.frame_w - pj // g.frame_w) <= wy) & (np.abs(pi % g.frame_w - pj % g.frame_w) <= wx)
+        else:
+            near = np.abs(pos_of(i, g) - pos_of(j, g)) <= pp.spatial_window
         return i_text | j_text | near
     if pattern == TEXTURAL:
         kept = j_text | in_checkerboard(j, g, pp.textural_stride)

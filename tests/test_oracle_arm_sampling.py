@@ -198,3 +198,28 @@ def test_spatial_recall_with_the_first_frame_as_key_frame(qk):
             kept2[a, b] = abs(strided[a] // G.S - strided[b] // G.S) <= 2 or strided[b] // G.S == 0     # floor(0.45 * 5) = 2
     assert Rs[0] == pytest.approx(expect, abs=1e-12)                                                  # floor(0.2 * 5) = 1 = PP's window
     assert Rs[1] == pytest.approx(recall_by_library(q, k, strided, kept2), abs=1e-12)
+
+
+def test_temporal_recall_with_a_2d_window(qk):
+    """The 2-D reading of the Temporal locality on both samples, rebuilt with loops and the library softmax."""
+    q, k = qk
+    wy, wx = 1, 2
+    pp2 = PatternParams(PP.frame_window, PP.spatial_window, PP.textural_stride, False, (wy, wx))
+
+    def kept_of(tokens):
+        n = len(tokens)
+        kept = np.zeros((n, n), dtype=bool)
+        for a in range(n):
+            for b in range(n):
+                pa, pb = tokens[a] % G.S, tokens[b] % G.S
+                kept[a, b] = abs(pa // G.frame_w - pb // G.frame_w) <= wy and abs(pa % G.frame_w - pb % G.frame_w) <= wx
+        return kept
+
+    first_frame = list(range(G.S))
+    strided = list(range(0, G.Nv, OMEGA))
+    _, (rt, rs, _), _ = orc.arm_head(q, k, G, pp2, orc.SAMPLE_ALG1, OMEGA, 0.9)
+    assert rt == pytest.approx(recall_by_library(q, k, first_frame, kept_of(first_frame)), abs=1e-12)
+    _, (rt_g, rs_g, _), _ = orc.arm_head(q, k, G, pp2, orc.SAMPLE_GLOBAL, OMEGA, 0.9)
+    assert rt_g == pytest.approx(recall_by_library(q, k, strided, kept_of(strided)), abs=1e-12)
+    _, (_, rs_plain, _), _ = orc.arm_head(q, k, G, PP, orc.SAMPLE_ALG1, OMEGA, 0.9)
+    assert rs == rs_g == rs_plain                      # the Spatial recall does not depend on it

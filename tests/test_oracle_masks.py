@@ -319,3 +319,60 @@ def test_key_first_frame_tile_lists_follow_the_mask():
             for b in range(nQ):
                 sub = kept[a * block:(a + 1) * block, b * block:(b + 1) * block]
                 assert (b in tiles) == bool(sub.any())
+
+
+# ---------------------------------------------------------------- Temporal head with a 2-D in-frame window
+
+def test_temporal_2d_window_by_enumeration():
+    """The other reading of Sec. 3.2's locality inside a frame: a window on rows and columns of the frame rather than a
+    band on the flattened index.  Nested loops over the definition; the other patterns do not change."""
+    g = Geometry(3, 4, 5, 2)
+    idx = np.arange(g.N)
+    for wy, wx in ((0, 0), (1, 2), (0, 4), (3, 0), (9, 9)):
+        pp = PatternParams(1, 2, 2, False, (wy, wx))
+        M = orc.keep_mask(TEMPORAL, idx, idx, g, pp)
+        for i in range(g.N):
+            for j in range(g.N):
+                if i >= g.Nv or j >= g.Nv:
+                    want = True
+                else:
+                    pi, pj = i % g.S, j % g.S
+                    want = abs(pi // g.frame_w - pj // g.frame_w) <= wy and abs(pi % g.frame_w - pj % g.frame_w) <= wx
+                assert M[i, j] == want, (wy, wx, i, j)
+        for pattern in (SPATIAL, TEXTURAL, DENSE):
+            assert np.array_equal(orc.keep_mask(pattern, idx, idx, g, pp), orc.keep_mask(pattern, idx, idx, g, PatternParams(1, 2, 2)))
+    # a window covering the frame keeps everything
+    assert orc.keep_mask(TEMPORAL, idx, idx, g, PatternParams(1, 0, 2, False, (3, 4))).all()
+
+
+def test_temporal_2d_window_is_a_kronecker_product_of_two_bands():
+    # video x video part = ones(T, T) (x) band_y(H) (x) band_x(W)
+    g = Geometry(3, 5, 6, 0)
+    wy, wx = 1, 2
+    idx = np.arange(g.N)
+    M = orc.keep_mask(TEMPORAL, idx, idx, g, PatternParams(0, 0, 2, False, (wy, wx)))
+    by = np.abs(np.subtract.outer(np.arange(g.frame_h), np.arange(g.frame_h))) <= wy
+    bx = np.abs(np.subtract.outer(np.arange(g.frame_w), np.arange(g.frame_w))) <= wx
+    assert np.array_equal(M, np.kron(np.ones((g.T, g.T), dtype=bool), np.kron(by, bx)))
+    # kept count: product of the two band counts, for every frame pair
+    cy = g.frame_h * (2 * wy + 1) - wy * (wy + 1)
+    cx = g.frame_w * (2 * wx + 1) - wx * (wx + 1)
+    assert M.sum() == g.T * g.T * cy * cx
+
+
+def test_temporal_2d_tile_lists_follow_the_mask():
+    g = Geometry(4, 6, 10, 7)
+    pp = PatternParams(1, 3, 2, False, (1, 3))
+    for permute in (False, True):
+        pq = orc.query_order(TEMPORAL, g, permute)
+        kept = orc.keep_mask(TEMPORAL, pq, pq, g, pp)
+        for block in (16, 64):
+            nQ = -(-g.N // block)
+            for a in range(0, nQ, 3):
+                row = orc.tile_row(TEMPORAL, g, pp, permute, block, block, a)
+                tiles = {e & ~orc.PARTIAL_BIT: bool(e & orc.PARTIAL_BIT) for e in row}
+                for b in range(nQ):
+                    sub = kept[a * block:(a + 1) * block, b * block:(b + 1) * block]
+                    assert (b in tiles) == bool(sub.any())
+                    if b in tiles:
+                        assert tiles[b] == (not (sub.all() and (b + 1) * block <= g.N))

@@ -82,6 +82,12 @@ typedef struct {
   int32_t spatial_key_first_frame; /* 0: a Spatial head keeps the frames within w_f (Eq. 3).  1: it keeps, in addition,
                                every key of frame 0 for every query: Sec. 3.2 lets the attended set hold adjacent
                                or key frames; the first frame is the one key frame offered here */
+  int32_t temporal_window_2d; /* 0: a Temporal head keeps the 1-D band |pos(q) - pos(k)| <= spatial_window.  1: it keeps
+                               the 2-D window |y(q) - y(k)| <= temporal_window_y and |x(q) - x(k)| <= temporal_window_x on
+                               the rows and columns of the frame instead (the other reading of Sec. 3.2's locality inside
+                               a frame; spatial_window is then unused).  Needs frame_h, frame_w < 32768; not available
+                               with the dynamic-bandwidth entry points (RF_ERR_UNSUPPORTED) */
+  int32_t temporal_window_y, temporal_window_x;   /* >= 0; read only when temporal_window_2d = 1 */
 } rf_params;
 
 /*

@@ -34,7 +34,8 @@ class rf_params(C.Structure):
     _fields_ = [("frame_window", C.c_int32), ("spatial_window", C.c_int32), ("textural_stride", C.c_int32),
                 ("sample_mode", C.c_int32), ("sample_stride", C.c_int32), ("alpha", C.c_float),
                 ("block_m", C.c_int32), ("block_n", C.c_int32), ("temporal_permute", C.c_int32),
-                ("two_mask", C.c_int32), ("spatial_key_first_frame", C.c_int32)]
+                ("two_mask", C.c_int32), ("spatial_key_first_frame", C.c_int32), ("temporal_window_2d", C.c_int32),
+                ("temporal_window_y", C.c_int32), ("temporal_window_x", C.c_int32)]
 
 
 class rf_schedule(C.Structure):
@@ -125,9 +126,12 @@ def make_shape(B, H, D, T, frame_h, frame_w, L_text) -> rf_shape:
 
 
 def make_params(frame_window, spatial_window, textural_stride=2, sample_mode=RF_SAMPLE_ALG1, sample_stride=1,
-                alpha=0.9, block_m=128, block_n=128, temporal_permute=1, two_mask=0, spatial_key_first_frame=0) -> rf_params:
+                alpha=0.9, block_m=128, block_n=128, temporal_permute=1, two_mask=0, spatial_key_first_frame=0,
+                temporal_window_2d=None) -> rf_params:
+    """temporal_window_2d: None, or (w_y, w_x) for the 2-D in-frame window of Temporal heads."""
+    t2 = (0, 0, 0) if temporal_window_2d is None else (1, int(temporal_window_2d[0]), int(temporal_window_2d[1]))
     return rf_params(frame_window, spatial_window, textural_stride, sample_mode, sample_stride, alpha,
-                     block_m, block_n, temporal_permute, two_mask, spatial_key_first_frame)
+                     block_m, block_n, temporal_permute, two_mask, spatial_key_first_frame, *t2)
 
 
 def shape_of(wl) -> rf_shape:
@@ -135,10 +139,12 @@ def shape_of(wl) -> rf_shape:
     return rf_shape(wl.B, wl.H, wl.D, wl.T, wl.frame_h, wl.frame_w, wl.L_text)
 
 
-def params_of(wl, block_m=128, block_n=128, temporal_permute=1, two_mask=0, spatial_key_first_frame=0) -> rf_params:
+def params_of(wl, block_m=128, block_n=128, temporal_permute=1, two_mask=0, spatial_key_first_frame=0,
+              temporal_window_2d=None) -> rf_params:
     """rf_params of a synth.Workload."""
     return rf_params(wl.frame_window, wl.spatial_window, wl.textural_stride, wl.sample_mode, wl.sample_stride,
-                     wl.alpha, block_m, block_n, temporal_permute, two_mask, spatial_key_first_frame)
+                     wl.alpha, block_m, block_n, temporal_permute, two_mask, spatial_key_first_frame,
+                     *((0, 0, 0) if temporal_window_2d is None else (1, int(temporal_window_2d[0]), int(temporal_window_2d[1]))))
 
 
 def rf_schedule_dims(shape: rf_shape, params: rf_params):

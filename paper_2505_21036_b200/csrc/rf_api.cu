@@ -11,6 +11,12 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
+// The kernels pack a frame row and column into one word for the 2-D Temporal window.
+rf_status check_2d(const rf_shape* s, const rf_params* p) {
+  if (p->temporal_window_2d == 1 && (s->frame_h >= 32768 || s->frame_w >= 32768)) return RF_ERR_UNSUPPORTED;
+  return RF_OK;
+}
+
 rf_status check_shape(const rf_shape* s) {
   if (s == nullptr) return RF_ERR_INVALID_ARG;
   if (s->B < 1 || s->H < 1 || s->T < 1 || s->frame_h < 1 || s->frame_w < 1 || s->L_text < 0) return RF_ERR_INVALID_ARG;
@@ -30,6 +36,8 @@ rf_status check_params(const rf_params* p) {
   if (p->temporal_permute != 0 && p->temporal_permute != 1) return RF_ERR_INVALID_ARG;
   if (p->two_mask != 0 && p->two_mask != 1) return RF_ERR_INVALID_ARG;
   if (p->spatial_key_first_frame != 0 && p->spatial_key_first_frame != 1) return RF_ERR_INVALID_ARG;
+  if (p->temporal_window_2d != 0 && p->temporal_window_2d != 1) return RF_ERR_INVALID_ARG;
+  if (p->temporal_window_2d == 1 && (p->temporal_window_y < 0 || p->temporal_window_x < 0)) return RF_ERR_INVALID_ARG;
   return RF_OK;
 }
 
@@ -64,12 +72,16 @@ RfGeom make_geom(const rf_shape* s, int wf, int ws, int tau, int bm, int bn, int
   g.permute = permute;
   g.two_mask = 0;
   g.key_first = 0;
+  g.t2d = g.wy = g.wx = 0;
   return g;
 }
 RfGeom make_geom(const rf_shape* s, const rf_params* p) {
   RfGeom g = make_geom(s, p->frame_window, p->spatial_window, p->textural_stride, p->block_m, p->block_n, p->temporal_permute);
   g.two_mask = p->two_mask;
   g.key_first = p->spatial_key_first_frame;
+  g.t2d = p->temporal_window_2d;
+  g.wy = g.t2d ? (p->temporal_window_y < g.Hf ? p->temporal_window_y : g.Hf) : 0;   // past the frame: same mask
+  g.wx = g.t2d ? (p->temporal_window_x < g.Wf ? p->temporal_window_x : g.Wf) : 0;
   return g;
 }
 
@@ -124,6 +136,8 @@ rf_status rf_checked_geom(const rf_shape* shape, const rf_params* params, RfGeom
   if (st != RF_OK) return st;
   st = check_params(params);
   if (st != RF_OK) return st;
+  st = check_2d(shape, params);
+  if (st != RF_OK) return st;
   *out = make_geom(shape, params);
   return RF_OK;
 }
@@ -138,6 +152,8 @@ rf_status sparse_attn_impl(const rf_shape* shape, const rf_params* params, const
   if (st != RF_OK) return st;
   st = check_params(params);
   if (st != RF_OK) return st;
+  st = check_2d(shape, params);
+  if (st != RF_OK) return st;
   if (params->block_m != 128 || params->block_n != 128) return RF_ERR_UNSUPPORTED;
   if (q == nullptr || k == nullptr || v == nullptr || o == nullptr || head_class == nullptr || sched == nullptr ||
       sched->count == nullptr || sched->kv_tile == nullptr || ws == nullptr)
@@ -145,6 +161,7 @@ rf_status sparse_attn_impl(const rf_shape* shape, const rf_params* params, const
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) ||
       (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0)
     return RF_ERR_INVALID_ARG;
+  if (head_window != nullptr && params->temporal_window_2d) return RF_ERR_UNSUPPORTED;
   if (ws_bytes < rf_workspace_bytes(shape, params)) return RF_ERR_WORKSPACE_TOO_SMALL;
   const RfGeom g = make_geom(shape, params);
   if (sched->nQ != g.nQ || sched->nKmax != g.nKmax) return RF_ERR_INVALID_ARG;
@@ -214,6 +231,8 @@ rf_status rf_schedule_dims(const rf_shape* shape, const rf_params* params, int32
   if (st != RF_OK) return st;
   st = check_params(params);
   if (st != RF_OK) return st;
+  st = check_2d(shape, params);
+  if (st != RF_OK) return st;
   const RfGeom g = make_geom(shape, params);
   if (nQ) *nQ = g.nQ;
   if (nKmax) *nKmax = g.nKmax;
@@ -233,6 +252,8 @@ rf_status rf_arm_classify(const rf_shape* shape, const rf_params* params, const 
   if (st != RF_OK) return st;
   st = check_params(params);
   if (st != RF_OK) return st;
+  st = check_2d(shape, params);
+  if (st != RF_OK) return st;
   if (shape->D != 64 && shape->D != 96 && shape->D != 128) return RF_ERR_UNSUPPORTED;
   if (q == nullptr || k == nullptr || head_class == nullptr || ws == nullptr) return RF_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return RF_ERR_INVALID_ARG;
@@ -250,6 +271,8 @@ rf_status rf_selftest_arm_abandoned(const rf_shape* shape, const rf_params* para
   rf_status st = check_shape(shape);
   if (st != RF_OK) return st;
   st = check_params(params);
+  if (st != RF_OK) return st;
+  st = check_2d(shape, params);
   if (st != RF_OK) return st;
   if (shape->D != 64 && shape->D != 96 && shape->D != 128) return RF_ERR_UNSUPPORTED;
   if (q == nullptr || k == nullptr || head_class == nullptr || ws == nullptr) return RF_ERR_INVALID_ARG;
@@ -271,7 +294,10 @@ rf_status rf_arm_classify_plus(const rf_shape* shape, const rf_params* params, c
   if (st != RF_OK) return st;
   st = check_params(params);
   if (st != RF_OK) return st;
+  st = check_2d(shape, params);
+  if (st != RF_OK) return st;
   if (shape->D != 64 && shape->D != 96 && shape->D != 128) return RF_ERR_UNSUPPORTED;
+  if (params->temporal_window_2d) return RF_ERR_UNSUPPORTED;   // a bandwidth has no 2-D meaning defined here
   if (bandwidths == nullptr || n_bandwidths < 1 || n_bandwidths > RF_MAX_BANDWIDTHS) return RF_ERR_INVALID_ARG;
   if (q == nullptr || k == nullptr || head_class == nullptr || head_window == nullptr || ws == nullptr) return RF_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0) return RF_ERR_INVALID_ARG;
@@ -303,6 +329,9 @@ rf_status rf_build_block_mask_plus(const rf_shape* shape, const rf_params* param
   if (st != RF_OK) return st;
   st = check_params(params);
   if (st != RF_OK) return st;
+  st = check_2d(shape, params);
+  if (st != RF_OK) return st;
+  if (head_window != nullptr && params->temporal_window_2d) return RF_ERR_UNSUPPORTED;
   if (head_class == nullptr || out == nullptr || out->count == nullptr || out->kv_tile == nullptr || out->kv_len == nullptr)
     return RF_ERR_INVALID_ARG;
   const RfGeom g = make_geom(shape, params);
@@ -346,6 +375,8 @@ rf_status rf_reorder_tokens(const rf_shape* shape, const rf_params* params, cons
   rf_status st = check_shape(shape);
   if (st != RF_OK) return st;
   st = check_params(params);
+  if (st != RF_OK) return st;
+  st = check_2d(shape, params);
   if (st != RF_OK) return st;
   if (q == nullptr || k == nullptr || v == nullptr || head_class == nullptr || ws == nullptr) return RF_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) != 0)

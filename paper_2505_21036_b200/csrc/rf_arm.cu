@@ -115,7 +115,8 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
   const CUtensorMap* map_q = &maps.q[which];
   const CUtensorMap* map_k = &maps.k[which];
   // positions equal sample indices only while the sample is contiguous and stays inside the first frame
-  const bool t_generic = sm.want_t && (stride != 1 || n > g.S);    // needs per-key positions
+  // (the 2-D in-frame window is not an interval of the sample index, so it always takes the per-key table)
+  const bool t_generic = sm.want_t && (stride != 1 || n > g.S || g.t2d);    // needs per-key positions
 
   if (tid == 0) {
     mbar_init(bar(C::B_Q), 1);
@@ -186,6 +187,7 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
       const int mc = min(m, n - 1);
       const int tok = mc * stride;
       const int rf = tok / g.S, rp = tok - rf * g.S;
+      const int ry = rp / g.Wf, rx = rp - ry * g.Wf;
       // Masks k = 0..NB-1: Temporal with window win.ws[k]; k = NB..2NB-1: Spatial with win.wf[k-NB];
       // k = 2NB: Textural.  Band masks keep one key interval [lo, hi) per row in sample-index space.
       constexpr int NM = 2 * NB + 1;
@@ -304,7 +306,7 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
                   const int ktok = min(u0 + c, n - 1) * stride;
                   const int kp = ktok % g.S;
                   const int y = kp / g.Wf, x = kp - y * g.Wf;
-                  attr_p[c] = kp;
+                  attr_p[c] = g.t2d ? ((y << 16) | x) : kp;    // frame dimensions stay below 2^15 with the 2-D window
                   attr_c[c] = (y % g.tau) == (x % g.tau);
                 }
                 __syncwarp();
@@ -322,6 +324,9 @@ __global__ void __launch_bounds__(ARM_THREADS, 1) rf_arm_kernel(const __grid_con
                   bool keep;
                   if (is_x) {
                     keep = attr_c[q4 * 32 + c] != 0;
+                  } else if (g.t2d) {
+                    const int yx = attr_p[q4 * 32 + c];
+                    keep = abs((yx >> 16) - ry) <= g.wy && abs((yx & 0xffff) - rx) <= g.wx;
                   } else {
                     const int dp = attr_p[q4 * 32 + c] - rp;
                     keep = (dp < 0 ? -dp : dp) <= wk;

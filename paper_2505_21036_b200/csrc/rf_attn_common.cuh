@@ -29,12 +29,13 @@ __device__ __forceinline__ float ex2(float x) {
 // order) and the always-kept text slots [text0, lkv).  Kept compact on purpose: PARTIAL tiles are
 // rare, and a large rarely-run code block costs more in instruction fetch than in arithmetic.
 struct RowMask {
-  int lo, hi;        // kept video slots [lo, hi) when !periodic
+  int lo, hi;        // kRange: kept video slots [lo, hi)
   int first_end;     // slots [0, first_end) are kept as well (Spatial with the first frame as key frame), else 0
   int text0;         // first always-kept (text) slot
   int lkv;           // number of key slots
-  int p, ws, S, T;   // periodic form: |slot % S - p| <= ws for slots of frames 0..T-1
-  bool periodic;
+  int p, ws, S, T;   // kPeriodic: |slot % S - p| <= ws for slots of frames 0..T-1
+  uint8_t mode;      // kRange: [lo, hi) and [0, first_end); kPeriodic: p +- ws in every frame; kWindow2d: see window2d_bits
+  enum : uint8_t { kRange = 0, kPeriodic = 1, kWindow2d = 2 };
 
   static __device__ __forceinline__ uint32_t below(int n) {  // bits [0, n) set, n in [0, 32]
     return n >= 32 ? 0xffffffffu : ((1u << n) - 1u);
@@ -50,9 +51,32 @@ struct RowMask {
       w[k] |= below(hi_k) & ~below(lo_k);
     }
   }
+  // mode == kWindow2d, a Temporal head with the 2-D in-frame window: the kept positions of query position
+  // p = y*W + x are, for each frame row y' within wy of y, the run [y'*W + x - wx, y'*W + x + wx] clipped to the row.
+  // In position-major order a position is T consecutive slots; in original order it recurs in every frame.  Only the
+  // rows the tile reaches are visited.  The fields the other modes use carry the frame's width and the window:
+  // lo = W, hi = wy, first_end = wx.
+  __device__ __forceinline__ void window2d_bits(int u0, uint32_t (&w)[4]) const {
+    const int W = lo, H = S / W, wy = hi, wx = first_end;
+    const int yq = p / W, xq = p - yq * W;
+    const int xlo = max(xq - wx, 0), xhi = min(xq + wx, W - 1);
+    const int ylo = max(yq - wy, 0), yhi = min(yq + wy, H - 1);
+    if (ws) {  // position-major slots
+      const int pa = u0 / T, pb = min((u0 + BN - 1) / T, S - 1);                   // positions the tile reaches
+      for (int y = max(ylo, pa / W); y <= min(yhi, pb / W); ++y) add(w, u0, (y * W + xlo) * T, (y * W + xhi + 1) * T);
+    } else {
+      const int f1 = min((u0 + BN - 1) / S, T - 1);
+      for (int f = u0 / S; f <= f1; ++f) {
+        const int pa = max(u0 - f * S, 0), pb = min(u0 + BN - 1 - f * S, S - 1);   // positions of frame f the tile reaches
+        for (int y = max(ylo, pa / W); y <= min(yhi, pb / W); ++y) add(w, u0, f * S + y * W + xlo, f * S + y * W + xhi + 1);
+      }
+    }
+  }
   __device__ __noinline__ void tile_bits(int u0, uint32_t (&w)[4]) const {
     w[0] = w[1] = w[2] = w[3] = 0u;
-    if (periodic) {
+    if (mode == kWindow2d) {
+      window2d_bits(u0, w);
+    } else if (mode == kPeriodic) {
       const int f1 = min((u0 + BN - 1) / S, T - 1);
       for (int f = u0 / S; f <= f1; ++f) add(w, u0, f * S + max(p - ws, 0), f * S + min(p + ws, S - 1) + 1);
     } else {
@@ -71,7 +95,7 @@ __device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r
   m.hi = m.lkv;
   m.first_end = 0;
   m.p = 0; m.ws = g.ws; m.S = g.S; m.T = g.T;
-  m.periodic = false;
+  m.mode = RowMask::kRange;
   if ((cls == RF_SPATIAL || cls == RF_TEMPORAL) && r < g.Nv) {
     m.text0 = g.Nv;
     if (cls == RF_SPATIAL) {
@@ -79,12 +103,17 @@ __device__ __forceinline__ RowMask make_row_mask(const RfGeom& g, int cls, int r
       m.lo = max(0, f - g.wf) * g.S;
       m.hi = min(g.T, f + g.wf + 1) * g.S;
       m.first_end = g.key_first ? g.S : 0;
+    } else if (g.t2d) {
+      m.mode = RowMask::kWindow2d;
+      m.p = g.permute ? r / g.T : r % g.S;
+      m.lo = g.Wf; m.hi = g.wy; m.first_end = g.wx;
+      m.ws = g.permute;
     } else if (g.permute) {
       const int p = r / g.T;
       m.lo = max(0, p - g.ws) * g.T;
       m.hi = min(g.S, p + g.ws + 1) * g.T;
     } else {
-      m.periodic = true;
+      m.mode = RowMask::kPeriodic;
       m.p = r % g.S;
     }
   }

@@ -22,6 +22,7 @@ struct RfGeom {
   int permute;           // Temporal heads in position-major order
   int two_mask;          // ARM decides between Spatial and Temporal only (ablation of Sec. 4.4)
   int key_first;         // Spatial heads also keep every key of frame 0 (a key frame, Sec. 3.2)
+  int t2d, wy, wx;       // Temporal heads keep the 2-D in-frame window |dy| <= wy, |dx| <= wx instead of the band ws
 };
 
 // Device-side error reporting: first error wins, kernels never trap.

@@ -21,6 +21,32 @@ __device__ __forceinline__ int cyclic_intervals(int a0, int a1, int S, Iv out[2]
   return 2;
 }
 
+// 2-D in-frame window between two runs of consecutive positions A = [a0, a1] and B = [b0, b1] (row-major positions
+// of a frame of width W): `any` - some pair (p in A, p' in B) has |dy| <= wy and |dx| <= wx; `all` - every pair has.
+// A run of positions is up to three rectangles (a partial first row, whole rows, a partial last row); between two
+// rectangles the smallest and largest |dy| and |dx| follow from the interval ends.
+struct Rect { int y0, y1, x0, x1; };
+__device__ __forceinline__ int run_rects(int p0, int p1, int W, Rect out[3]) {
+  const int ya = p0 / W, xa = p0 - ya * W, yb = p1 / W, xb = p1 - yb * W;
+  if (ya == yb) { out[0] = {ya, ya, xa, xb}; return 1; }
+  int n = 0;
+  out[n++] = {ya, ya, xa, W - 1};
+  if (yb - ya > 1) out[n++] = {ya + 1, yb - 1, 0, W - 1};
+  out[n++] = {yb, yb, 0, xb};
+  return n;
+}
+__device__ void window2d(const Iv& A, const Iv& B, int W, int wy, int wx, bool& any, bool& all) {
+  Rect ra[3], rb[3];
+  const int na = run_rects(A.lo, A.hi, W, ra), nb = run_rects(B.lo, B.hi, W, rb);
+  for (int i = 0; i < na; ++i)
+    for (int j = 0; j < nb; ++j) {
+      const int gy = max(max(rb[j].y0 - ra[i].y1, ra[i].y0 - rb[j].y1), 0), gx = max(max(rb[j].x0 - ra[i].x1, ra[i].x0 - rb[j].x1), 0);
+      const int sy = max(ra[i].y1 - rb[j].y0, rb[j].y1 - ra[i].y0), sx = max(ra[i].x1 - rb[j].x0, rb[j].x1 - ra[i].x0);
+      any = any || (gy <= wy && gx <= wx);
+      all = all && (sy <= wy && sx <= wx);
+    }
+}
+
 // 0: empty, 1: PARTIAL, 2: FULL.  Tile (a, b) of a head of class cls.
 __device__ int tile_flag(const RfGeom& g, int cls, int a, int b) {
   const int Lkv = rf_kv_len(g, cls);
@@ -36,7 +62,22 @@ __device__ int tile_flag(const RfGeom& g, int cls, int a, int b) {
     bool vv_any = false, vv_all = true;
     if (video_part) {
       const int rv1 = min(r1, Nv), uv1 = min(u1, Nv);
-      if (cls == RF_SPATIAL || g.permute) {
+      if (cls == RF_TEMPORAL && g.t2d) {
+        // 2-D in-frame window: the tile's query and key slots each cover one run of positions (position-major
+        // order) or a run that may wrap round the frame's end (original order)
+        Iv R[2], C[2];
+        int nr, nc;
+        if (g.permute) {
+          R[0] = {r0 / g.T, (rv1 - 1) / g.T};
+          C[0] = {u0 / g.T, (uv1 - 1) / g.T};
+          nr = nc = 1;
+        } else {
+          nr = cyclic_intervals(r0, rv1, g.S, R);
+          nc = cyclic_intervals(u0, uv1, g.S, C);
+        }
+        for (int i = 0; i < nr; ++i)
+          for (int j = 0; j < nc; ++j) window2d(R[i], C[j], g.Wf, g.wy, g.wx, vv_any, vv_all);
+      } else if (cls == RF_SPATIAL || g.permute) {
         // contiguous ranges of frames (Spatial) or of positions (position-major Temporal)
         const int unit = cls == RF_SPATIAL ? g.S : g.T;
         const int w = cls == RF_SPATIAL ? g.wf : g.ws;

@@ -18,8 +18,9 @@ def geom(wl):
     return orc.Geometry(wl.T, wl.frame_h, wl.frame_w, wl.L_text)
 
 
-def pparams(wl, key_first=False):
-    return orc.PatternParams(wl.frame_window, wl.spatial_window, wl.textural_stride, bool(key_first))
+def pparams(wl, key_first=False, t2d=None):
+    return orc.PatternParams(wl.frame_window, wl.spatial_window, wl.textural_stride, bool(key_first),
+                             None if t2d is None else tuple(t2d))
 
 
 def to_dev(bits: np.ndarray) -> torch.Tensor:
@@ -68,12 +69,12 @@ class Run:
     (classes, recalls, schedule arrays, workspace, outputs) sits between guard words that are checked after
     every call."""
 
-    def __init__(self, wl, qkv=None, block=128, temporal_permute=1, two_mask=0, key_first=0):
+    def __init__(self, wl, qkv=None, block=128, temporal_permute=1, two_mask=0, key_first=0, t2d=None):
         self.wl = wl
         self.q_bits, self.k_bits, self.v_bits = qkv if qkv is not None else synth.make_qkv(wl)
         self.q, self.k, self.v = (to_dev(x) for x in (self.q_bits, self.k_bits, self.v_bits))
         self.shape = api.shape_of(wl)
-        self.params = api.params_of(wl, block, block, temporal_permute, two_mask, key_first)
+        self.params = api.params_of(wl, block, block, temporal_permute, two_mask, key_first, t2d)
         self.mem = Guarded()
         self.ws = self.mem.alloc((api.rf_workspace_bytes(self.shape, self.params),), torch.uint8, name="ws")
         self.sched = api.Schedule(self.shape, self.params, "cuda", with_bitmap=True)
@@ -185,8 +186,8 @@ def check_attention(O_gpu, lse_gpu, O_ref, lse_ref, what="", strict=True):
     return err.max(), err.mean(), rel, lerr
 
 
-def oracle_lists(wl, cls, block, permute, tiles=None, key_first=False):
-    g, pp = geom(wl), pparams(wl, key_first)
+def oracle_lists(wl, cls, block, permute, tiles=None, key_first=False, t2d=None):
+    g, pp = geom(wl), pparams(wl, key_first, t2d)
     nQ = -(-g.N // block)
     tiles = range(nQ) if tiles is None else tiles
     return {a: orc.tile_row(cls, g, pp, bool(permute), block, block, a) for a in tiles}

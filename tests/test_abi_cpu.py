@@ -53,7 +53,8 @@ def test_schedule_dims_and_workspace_for_every_workload(lib):
 @pytest.mark.parametrize("field,value", [("frame_window", -1), ("spatial_window", -1), ("textural_stride", 0),
                                          ("sample_stride", 0), ("sample_mode", 2), ("alpha", 0.0), ("alpha", 1.5),
                                          ("block_m", 48), ("block_n", 8), ("temporal_permute", 2), ("two_mask", 2),
-                                         ("two_mask", -1), ("spatial_key_first_frame", 2), ("spatial_key_first_frame", -1)])
+                                         ("two_mask", -1), ("spatial_key_first_frame", 2), ("spatial_key_first_frame", -1),
+                                         ("temporal_window_2d", 2), ("temporal_window_2d", -1)])
 def test_bad_parameters_are_rejected(lib, field, value):
     wl = synth.WORKLOADS["tiny"]
     s, p = api.shape_of(wl), api.params_of(wl)
@@ -130,3 +131,22 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(api, "_LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(api.RainFusionError):
         api.load()
+
+
+def test_2d_temporal_window_parameters(lib):
+    """The 2-D window's half-widths are checked only when the option is on, any non-negative value is accepted (a window
+    past the frame keeps every key), and the dynamic-bandwidth classifier refuses the combination before touching memory."""
+    wl = synth.WORKLOADS["tiny"]
+    s = api.shape_of(wl)
+    off = api.params_of(wl)
+    off.temporal_window_y = -5
+    assert lib.rf_workspace_bytes(C.byref(s), C.byref(off)) > 0
+    on = api.params_of(wl, temporal_window_2d=(1, 10 ** 6))
+    assert (on.temporal_window_2d, on.temporal_window_y, on.temporal_window_x) == (1, 1, 10 ** 6)
+    assert lib.rf_workspace_bytes(C.byref(s), C.byref(on)) == lib.rf_workspace_bytes(C.byref(s), C.byref(api.params_of(wl)))
+    for field in ("temporal_window_y", "temporal_window_x"):
+        bad = api.params_of(wl, temporal_window_2d=(1, 1))
+        setattr(bad, field, -1)
+        assert lib.rf_workspace_bytes(C.byref(s), C.byref(bad)) == 0
+    bw = (C.c_float * 2)(0.2, 0.5)
+    assert lib.rf_arm_classify_plus(C.byref(s), C.byref(on), bw, 2, None, None, None, None, None, None, 0, None, None) != 0

@@ -500,3 +500,46 @@ def test_first_frame_as_key_frame(mode):
             small.build()
             ref = gu.oracle_lists(wl, S_, block, 1, key_first=True)
             assert small.lists(0, 0) == [ref[a] for a in range(small.sched.nQ)], (kw, block)
+
+
+# ------------------------------------------------------------------ Temporal heads with a 2-D in-frame window
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("permute", [0, 1])
+def test_temporal_2d_window(mode, permute):
+    """The other reading of Sec. 3.2's locality for Temporal heads: a query keeps the keys whose in-frame row and column
+    both lie within a window of its own, in every frame.  ARM's Temporal recall under both sampling modes, the tile lists
+    at several tile sizes in both slot orders and the attention output against the oracle; the other patterns must not
+    change, and the dynamic-bandwidth entry points refuse the combination."""
+    for kw, t2d in ((dict(T=6, fh=12, fw=11, L=37, wf=1, ws=20, omega=6), (2, 3)),
+                    (dict(T=9, fh=5, fw=8, L=0, wf=0, ws=3, omega=7), (0, 2)),
+                    (dict(T=4, fh=20, fw=20, L=9, wf=2, ws=50, omega=3), (4, 1)),
+                    (dict(T=3, fh=17, fw=23, L=5, wf=1, ws=9, omega=4), (40, 50))):      # a window past the frame: every key
+        wl = synth.small_workload("t2d", H=4, D=64, mode=mode, amp=1.5, **kw)
+        g, pp = gu.geom(wl), gu.pparams(wl, t2d=t2d)
+        run = gu.Run(wl, temporal_permute=permute, t2d=t2d)
+        cls_gpu, rec_gpu = run.arm()
+        cls_ref, rec_ref, margin = orc.arm_classify(run.q_bits, run.k_bits, g, pp, wl.sample_mode, wl.sample_stride, wl.alpha)
+        assert np.abs(rec_gpu - rec_ref).max() <= gu.RECALL_ABS, (kw, np.abs(rec_gpu - rec_ref).max())
+        decided = margin > gu.TIE_MARGIN
+        assert np.array_equal(cls_gpu[decided], cls_ref[decided])
+        plain = gu.Run(wl, temporal_permute=permute)
+        _, rec_plain = plain.arm()
+        assert np.allclose(rec_gpu[..., 1:], rec_plain[..., 1:], atol=1e-6)       # Spatial and Textural recalls untouched
+        classes = [S_, T_, X_, D_]
+        run.force_classes(classes)
+        run.build()
+        O, lse = run.sparse()
+        for h, cls in enumerate(classes):
+            ref = gu.oracle_lists(wl, cls, 128, permute, t2d=t2d)
+            assert run.lists(0, h) == [ref[a] for a in range(run.sched.nQ)], (kw, cls)
+            Or, lr = orc.masked_attention(run.q_bits[0, h], run.k_bits[0, h], run.v_bits[0, h], cls, g, pp)
+            gu.check_attention(O[0, h], lse[0, h], Or, lr, f"2-D temporal window {kw}, class {cls}", strict=False)
+        for block in (16, 32, 64):
+            small = gu.Run(wl, block=block, temporal_permute=permute, t2d=t2d)
+            small.force_classes(classes)
+            small.build()
+            ref = gu.oracle_lists(wl, T_, block, permute, t2d=t2d)
+            assert small.lists(0, 1) == [ref[a] for a in range(small.sched.nQ)], (kw, block)
+        with pytest.raises(api.RainFusionError, match="unsupported"):
+            run.arm_plus([0.2, 0.5])

@@ -47,9 +47,21 @@ def test_random_case_up_to_forty_tiles(seed):
     check_case(seed, *draw_case(seed, large=True))
 
 
-def check_case(seed, wl, permute, two_mask, classes):
-    g, pp = gu.geom(wl), gu.pparams(wl)
-    run = gu.Run(wl, temporal_permute=permute, two_mask=two_mask)
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("RF_FUZZ_OPT_FROM", "0")),
+                                       int(__import__("os").environ.get("RF_FUZZ_OPT_TO", "16"))))
+def test_random_case_pattern_options(seed):
+    """The optional readings of Sec. 3.2 on drawn shapes: the first frame as a key frame of Spatial heads, a 2-D
+    in-frame window for Temporal heads, or both."""
+    wl, permute, two_mask, classes = draw_case(5000 + seed, large=seed % 4 == 3)
+    rng = np.random.default_rng(31000 + seed)
+    which = int(rng.integers(1, 4))
+    t2d = (int(rng.integers(0, wl.frame_h + 2)), int(rng.integers(0, wl.frame_w + 2))) if which & 2 else None
+    check_case(seed, wl, permute, two_mask, classes, key_first=which & 1, t2d=t2d)
+
+
+def check_case(seed, wl, permute, two_mask, classes, key_first=0, t2d=None):
+    g, pp = gu.geom(wl), gu.pparams(wl, key_first, t2d)
+    run = gu.Run(wl, temporal_permute=permute, two_mask=two_mask, key_first=key_first, t2d=t2d)
     # ARM
     cls_gpu, rec_gpu = run.arm()
     cls_ref, rec_ref, margin = orc.arm_classify(run.q_bits, run.k_bits, g, pp, wl.sample_mode, wl.sample_stride, wl.alpha,
@@ -64,19 +76,19 @@ def check_case(seed, wl, permute, two_mask, classes):
     for b in range(wl.B):
         for h in range(wl.H):
             cls = int(classes[b, h])
-            ref = gu.oracle_lists(wl, cls, 128, permute)
+            ref = gu.oracle_lists(wl, cls, 128, permute, key_first=key_first, t2d=t2d)
             assert run.lists(b, h) == [ref[a] for a in range(run.sched.nQ)], (seed, b, h, cls)
             assert int(run.sched.kv_len[b, h]) == orc.kv_len(cls, g, pp)
             Or, lr = orc.masked_attention(run.q_bits[b, h], run.k_bits[b, h], run.v_bits[b, h], cls, g, pp)
             gu.check_attention(O[b, h], lse[b, h], Or, lr, f"fuzz {seed} b{b} h{h} class {cls}", strict=False)
     # the schedule builder alone at a smaller tile (the attention kernel itself only takes 128 x 128)
     block = (16, 32, 64)[seed % 3]
-    small = gu.Run(wl, block=block, temporal_permute=permute)
+    small = gu.Run(wl, block=block, temporal_permute=permute, key_first=key_first, t2d=t2d)
     small.force_classes(classes)
     small.build()
     for b in range(wl.B):
         for h in range(wl.H):
-            ref = gu.oracle_lists(wl, int(classes[b, h]), block, permute)
+            ref = gu.oracle_lists(wl, int(classes[b, h]), block, permute, key_first=key_first, t2d=t2d)
             assert small.lists(b, h) == [ref[a] for a in range(small.sched.nQ)], (seed, b, h, block)
     if seed % 4 == 0:
         Od, lsed = run.dense()

@@ -82,7 +82,7 @@ class ClockSampler:
         self.tmp.flush()
         rows = [l.strip().split(", ") for l in open(self.tmp.name) if l.strip()]
         os.unlink(self.tmp.name)
-        sm, reasons, mx = [], set(), None
+        sm, pw, reasons, mx = [], [], set(), None
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             if len(r) < 7:
@@ -92,11 +92,19 @@ class ClockSampler:
                 mx = float(r[1])
             except ValueError:
                 continue
+            try:
+                pw.append(float(r[2]))
+            except ValueError:
+                pass
             for n, val in zip(names, r[3:7]):
                 if val.strip().lower().startswith("active"):
                     reasons.add(n)
         if sm:
             out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        if pw:
+            # board power over the same samples: with sw_power_cap among the reasons and the median at the board's limit
+            # the timed kernels are bound by power, and the SM clock is what the limit leaves
+            out.update(power_w=float(np.median(pw)), power_w_max=float(np.max(pw)))
         return out
 
 

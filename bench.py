@@ -56,7 +56,7 @@ def dense_flops(wl):
 class ClockSampler:
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
+             "clocks_event_reasons.sw_power_cap,power.draw.instant,power.limit")
 
     def __init__(self, gpu_id: str):
         """gpu_id: what `nvidia-smi -i` takes.  Pass the device's UUID ("GPU-..."): the CUDA ordinal is not the
@@ -82,7 +82,7 @@ class ClockSampler:
         self.tmp.flush()
         rows = [l.strip().split(", ") for l in open(self.tmp.name) if l.strip()]
         os.unlink(self.tmp.name)
-        sm, pw, reasons, mx = [], [], set(), None
+        sm, pw, reasons, mx, limit = [], [], set(), None, None
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             if len(r) < 7:
@@ -93,8 +93,10 @@ class ClockSampler:
             except ValueError:
                 continue
             try:
-                pw.append(float(r[2]))
-            except ValueError:
+                # power.draw is a one-second average on this generation: take the instantaneous reading
+                pw.append(float(r[7]))
+                limit = float(r[8])
+            except (ValueError, IndexError):
                 pass
             for n, val in zip(names, r[3:7]):
                 if val.strip().lower().startswith("active"):
@@ -104,7 +106,7 @@ class ClockSampler:
         if pw:
             # board power over the same samples: with sw_power_cap among the reasons and the median at the board's limit
             # the timed kernels are bound by power, and the SM clock is what the limit leaves
-            out.update(power_w=float(np.median(pw)), power_w_max=float(np.max(pw)))
+            out.update(power_w=float(np.median(pw)), power_w_max=float(np.max(pw)), power_limit_w=limit)
         return out
 
 

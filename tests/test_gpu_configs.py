@@ -176,6 +176,34 @@ def test_dynamic_bandwidth_at_full_size(name):
     check_rows(run, O, lse, cls_gpu, synth.sample_rows(wl, 256, seed=9), range(wl.H), pp_of_head)
 
 
+def test_pattern_options_at_full_size():
+    """The two optional readings of Sec. 3.2 at the OpenSoraPlan shape (D = 96, 86 700 tokens), both switched on: the
+    first frame as a key frame of Spatial heads and a 2-D in-frame window for Temporal heads.  ARM on every head, tile
+    lists on sampled query tiles, 256 rows per head of the attention, against the oracle."""
+    name = "opensoraplan"
+    wl = synth.WORKLOADS[name]
+    t2d = (wl.frame_h // 4, wl.frame_w // 4)
+    g, pp = gu.geom(wl), gu.pparams(wl, True, t2d)
+    run = gu.Run(wl, qkv=inputs(name), key_first=1, t2d=t2d)
+    cls_gpu, rec_gpu = run.arm()
+    cls_ref, rec_ref, margin = orc.arm_classify(run.q_bits, run.k_bits, g, pp, wl.sample_mode, wl.sample_stride, wl.alpha)
+    assert np.abs(rec_gpu - rec_ref).max() <= gu.RECALL_ABS
+    decided = margin > gu.TIE_MARGIN
+    assert np.array_equal(cls_gpu[decided], cls_ref[decided])
+    classes = np.asarray([S_, T_, X_] * (wl.H // 3), dtype=np.int32)   # every pattern, whatever ARM made of the options
+    run.force_classes(classes)
+    run.build()
+    tiles = sample_tiles(run.sched.nQ, k=6)
+    ref = {c: gu.oracle_lists(wl, c, 128, 1, tiles, key_first=True, t2d=t2d) for c in (S_, T_, X_)}
+    for h in range(wl.H):
+        got = run.lists(0, h)
+        for a in tiles:
+            assert got[a] == ref[int(classes[h])][a], (h, a)
+        assert int(run.sched.kv_len[0, h]) == orc.kv_len(int(classes[h]), g, pp)
+    O, lse = gpu_outputs(run)
+    check_rows(run, O, lse, classes, synth.sample_rows(wl, 256, seed=12), range(0, wl.H, 2), lambda h: pp)
+
+
 def test_two_mask_ablation_at_cogvideox_literal_amplitude():
     """Table 2's rows without the Textural mask at the CogVideoX shape with the planted amplitude its configuration
     states (0.5): neither recall reaches alpha for any head, so every head takes the mask of larger recall."""

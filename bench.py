@@ -262,7 +262,7 @@ def run_cuda(args, wl):
     # heads over a copy-in, a compute and a copy-out stream; the same kernels run as in the device-resident step.
     from paper_2505_21036_b200.layer import HostStagedAttention
     heads = wl.B * wl.H
-    groups = args.e2e_groups if args.e2e_groups > 0 else next(g for g in (4, 3, 2, 1) if heads % g == 0)
+    groups = args.e2e_groups if args.e2e_groups > 0 else next(g for g in (8, 6, 4, 3, 2, 1) if heads % g == 0)
     staged = HostStagedAttention(shape, params, dev, groups=groups)
 
     def e2e_step():

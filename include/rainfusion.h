@@ -232,11 +232,14 @@ rf_status rf_sparse_attn_fwd_plus(const rf_shape *shape, const rf_params *params
 /*
  * The whole path of Fig. 2a (ARM of Sec. 3.3 -> masks of Sec. 3.2 -> masked attention, Eq. 1-2) for callers whose
  * Q, K, V and O live in HOST memory.  Heads are independent at every stage (Algorithm 1 outputs one category per
- * head), so a run is pipelined over `head_groups` groups of heads (head_groups must divide B*H) on three streams of
- * the pipeline's own: copy-in, compute, copy-out.  Every byte of Q, K, V crosses to the device and every byte of O
- * comes back in every run; only the waiting overlaps, inside a run and between runs made back to back.
+ * head), so a run is pipelined over `head_groups` groups of heads (head_groups must divide B*H) on streams of the
+ * pipeline's own: copy-in, copy-out, and two compute streams that consecutive groups alternate on (so that one
+ * group's kernels fill the SMs the previous group's last CTAs leave).  Every byte of Q, K, V crosses to the device
+ * and every byte of O comes back in every run; only the waiting overlaps, inside a run and between runs made back
+ * to back.
  *   rf_host_pipeline_staging_bytes  host, pure: device bytes the pipeline needs (staged Q, K, V, O for all heads,
- *                                   workspace and schedule of one group, classes, status).  0 on bad arguments.
+ *                                   workspace and schedule of one group per compute stream, classes, status).
+ *                                   0 on bad arguments.
  *   rf_host_pipeline_create         staging: device memory of at least that size, 256-byte aligned, owned by the caller
  *                                   and handed to the pipeline until it is destroyed.  Creates streams and events only.
  *   rf_host_pipeline_run            q/k/v/o_host: host bf16 [B,H,N,D], pinned for the copies to overlap; the inputs

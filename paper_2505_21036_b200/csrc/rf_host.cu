@@ -5,7 +5,10 @@
 // ARM -> tile schedule -> masked attention runs, the next group's inputs arrive from the host and the previous
 // group's output leaves.  Every byte of Q, K, V still crosses to the device and every byte of O comes back in every
 // call; only the waiting overlaps.  Calls made back to back overlap as well: a group's staging buffers are refilled
-// for the next call as soon as this call's kernels have read them.
+// for the next call as soon as this call's kernels have read them.  Consecutive groups compute on two alternating
+// streams, each with a workspace and schedule arrays of its own: the last CTAs of one group's attention kernel
+// (a CTA runs for about a millisecond at the large shapes) then leave their SMs to the next group's kernels instead
+// of to nobody.
 // The pipeline object holds streams and events only; device memory comes from the caller in one block.
 #include <new>
 #include <vector>
@@ -18,12 +21,13 @@ struct rf_host_pipeline {
   int groups, heads_per_group;
   size_t head_elems;            // N * D
   __nv_bfloat16 *q, *k, *v, *o; // staging, [B*H, N, D]
-  uint8_t* ws;                  // workspace of one group (groups run one after the other on the compute stream)
+  int lanes;                    // compute streams in use: 2, or 1 when there is a single group
+  uint8_t* ws[2];               // workspace of one group, per compute stream
   size_t ws_bytes;
-  rf_schedule sched;            // schedule arrays of one group
+  rf_schedule sched[2];         // schedule arrays of one group, per compute stream
   int32_t* head_class;          // [groups, heads_per_group]
   int32_t* status;
-  cudaStream_t s_in, s_run, s_out;
+  cudaStream_t s_in, s_run[2], s_out;
   std::vector<cudaEvent_t> landed, run_done, out_done;
   cudaEvent_t all_done;
   bool ran;
@@ -56,7 +60,8 @@ bool layout_of(const rf_shape* shape, const rf_params* params, int groups, rf_sh
   L->kv_len = align_up((size_t)gshape->H * sizeof(int32_t));
   L->head_class = align_up((size_t)heads * sizeof(int32_t));
   L->status = kAlign;
-  L->total = 4 * L->tensor + L->ws + L->count + L->kv_tile + L->kv_len + L->head_class + L->status;
+  const size_t lanes = groups > 1 ? 2 : 1;
+  L->total = 4 * L->tensor + lanes * (L->ws + L->count + L->kv_tile + L->kv_len) + L->head_class + L->status;
   return true;
 }
 
@@ -67,7 +72,8 @@ void destroy(rf_host_pipeline* p) {
       if (e) cudaEventDestroy(e);
   if (p->all_done) cudaEventDestroy(p->all_done);
   if (p->s_in) cudaStreamDestroy(p->s_in);
-  if (p->s_run) cudaStreamDestroy(p->s_run);
+  for (cudaStream_t st : p->s_run)
+    if (st) cudaStreamDestroy(st);
   if (p->s_out) cudaStreamDestroy(p->s_out);
   delete p;
 }
@@ -108,28 +114,33 @@ rf_status rf_host_pipeline_create(const rf_shape* shape, const rf_params* params
   p->k = reinterpret_cast<__nv_bfloat16*>(b); b += L.tensor;
   p->v = reinterpret_cast<__nv_bfloat16*>(b); b += L.tensor;
   p->o = reinterpret_cast<__nv_bfloat16*>(b); b += L.tensor;
-  p->ws = b; p->ws_bytes = L.ws; b += L.ws;
-  p->sched.count = reinterpret_cast<int32_t*>(b); b += L.count;
-  p->sched.kv_tile = reinterpret_cast<int32_t*>(b); b += L.kv_tile;
-  p->sched.kv_len = reinterpret_cast<int32_t*>(b); b += L.kv_len;
-  p->sched.bitmap = nullptr;
-  p->sched.nQ = nQ;
-  p->sched.nKmax = nK;
+  p->lanes = head_groups > 1 ? 2 : 1;
+  p->ws_bytes = L.ws;
+  for (int r = 0; r < p->lanes; ++r) {
+    p->ws[r] = b; b += L.ws;
+    p->sched[r].count = reinterpret_cast<int32_t*>(b); b += L.count;
+    p->sched[r].kv_tile = reinterpret_cast<int32_t*>(b); b += L.kv_tile;
+    p->sched[r].kv_len = reinterpret_cast<int32_t*>(b); b += L.kv_len;
+    p->sched[r].bitmap = nullptr;
+    p->sched[r].nQ = nQ;
+    p->sched[r].nKmax = nK;
+  }
   p->head_class = reinterpret_cast<int32_t*>(b); b += L.head_class;
   p->status = reinterpret_cast<int32_t*>(b);
-  p->s_in = p->s_run = p->s_out = nullptr;
+  p->s_in = p->s_run[0] = p->s_run[1] = p->s_out = nullptr;
   p->all_done = nullptr;
   p->ran = false;
   bool ok = cudaStreamCreateWithFlags(&p->s_in, cudaStreamNonBlocking) == cudaSuccess &&
-            cudaStreamCreateWithFlags(&p->s_run, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&p->s_run[0], cudaStreamNonBlocking) == cudaSuccess &&
+            (p->lanes < 2 || cudaStreamCreateWithFlags(&p->s_run[1], cudaStreamNonBlocking) == cudaSuccess) &&
             cudaStreamCreateWithFlags(&p->s_out, cudaStreamNonBlocking) == cudaSuccess &&
             cudaEventCreateWithFlags(&p->all_done, cudaEventDisableTiming) == cudaSuccess;
   for (auto* vec : {&p->landed, &p->run_done, &p->out_done}) {
     vec->assign(head_groups, nullptr);
     for (int g = 0; ok && g < head_groups; ++g) ok = cudaEventCreateWithFlags(&(*vec)[g], cudaEventDisableTiming) == cudaSuccess;
   }
-  ok = ok && cudaMemsetAsync(p->status, 0, sizeof(int32_t), p->s_run) == cudaSuccess &&
-       cudaStreamSynchronize(p->s_run) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(p->status, 0, sizeof(int32_t), p->s_run[0]) == cudaSuccess &&
+       cudaStreamSynchronize(p->s_run[0]) == cudaSuccess;
   if (!ok) {
     destroy(p);
     return RF_ERR_CUDA;
@@ -141,7 +152,7 @@ rf_status rf_host_pipeline_create(const rf_shape* shape, const rf_params* params
 void rf_host_pipeline_destroy(rf_host_pipeline* p) {
   if (p == nullptr) return;
   cudaStreamSynchronize(p->s_in);
-  cudaStreamSynchronize(p->s_run);
+  for (int r = 0; r < p->lanes; ++r) cudaStreamSynchronize(p->s_run[r]);
   cudaStreamSynchronize(p->s_out);
   destroy(p);
 }
@@ -163,18 +174,20 @@ rf_status rf_host_pipeline_run(rf_host_pipeline* p, const void* q_host, const vo
     RF_TRY(cudaEventRecord(p->landed[g], p->s_in));
   }
   for (int g = 0; g < p->groups; ++g) {
-    RF_TRY(cudaStreamWaitEvent(p->s_run, p->landed[g], 0));
+    const int r = g % p->lanes;
+    cudaStream_t run = p->s_run[r];
+    RF_TRY(cudaStreamWaitEvent(run, p->landed[g], 0));
     // the previous call's output of this group has left the staging buffer
-    if (p->ran) RF_TRY(cudaStreamWaitEvent(p->s_run, p->out_done[g], 0));
+    if (p->ran) RF_TRY(cudaStreamWaitEvent(run, p->out_done[g], 0));
     int32_t* hc = p->head_class + (size_t)g * p->heads_per_group;
     const __nv_bfloat16 *q = p->q + g * gelems, *k = p->k + g * gelems, *v = p->v + g * gelems;
-    rf_status st = rf_arm_classify(&p->gshape, &p->params, q, k, hc, nullptr, p->ws, p->ws_bytes, p->status, p->s_run);
-    if (st == RF_OK) st = rf_build_block_mask(&p->gshape, &p->params, hc, &p->sched, p->status, p->s_run);
+    rf_status st = rf_arm_classify(&p->gshape, &p->params, q, k, hc, nullptr, p->ws[r], p->ws_bytes, p->status, run);
+    if (st == RF_OK) st = rf_build_block_mask(&p->gshape, &p->params, hc, &p->sched[r], p->status, run);
     if (st == RF_OK)
-      st = rf_sparse_attn_fwd(&p->gshape, &p->params, q, k, v, hc, &p->sched, p->o + g * gelems, nullptr, p->ws, p->ws_bytes,
-                              p->status, p->s_run);
+      st = rf_sparse_attn_fwd(&p->gshape, &p->params, q, k, v, hc, &p->sched[r], p->o + g * gelems, nullptr, p->ws[r],
+                              p->ws_bytes, p->status, run);
     if (st != RF_OK) return st;
-    RF_TRY(cudaEventRecord(p->run_done[g], p->s_run));
+    RF_TRY(cudaEventRecord(p->run_done[g], run));
     RF_TRY(cudaStreamWaitEvent(p->s_out, p->run_done[g], 0));
     RF_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(o_host) + (size_t)g * gbytes, p->o + g * gelems, gbytes, cudaMemcpyDeviceToHost,
                            p->s_out));

@@ -150,3 +150,38 @@ def test_2d_temporal_window_parameters(lib):
         assert lib.rf_workspace_bytes(C.byref(s), C.byref(bad)) == 0
     bw = (C.c_float * 2)(0.2, 0.5)
     assert lib.rf_arm_classify_plus(C.byref(s), C.byref(on), bw, 2, None, None, None, None, None, None, 0, None, None) != 0
+
+
+def test_header_from_plain_c_matches_the_binding(lib, tmp_path):
+    """The header compiles as strict C99, a C program links against the library, and what it sees (structure sizes and
+    field offsets, the results of the host-only entry points) is what the ctypes binding holds and returns."""
+    import os
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    libdir, exe = os.path.dirname(api.lib_path()), str(tmp_path / "abi_probe")
+    cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(root, "include"),
+           os.path.join(root, "tests", "abi_probe.c"), "-o", exe, "-L", libdir, "-l:" + os.path.basename(api.lib_path()),
+           "-Wl,-rpath," + libdir]
+    subprocess.run(cmd, check=True, capture_output=True, text=True)
+    out = subprocess.run([exe], check=True, capture_output=True, text=True).stdout
+    seen = dict(line.split(" ", 1) for line in out.strip().splitlines())
+    for name, struct in (("rf_shape", api.rf_shape), ("rf_params", api.rf_params), ("rf_schedule", api.rf_schedule)):
+        assert int(seen[f"sizeof.{name}"]) == C.sizeof(struct), name
+        fields = [f[0] for f in struct._fields_]
+        assert sorted(k.split(".")[2] for k in seen if k.startswith(f"offsetof.{name}.")) == sorted(fields), name
+        for f in fields:
+            assert int(seen[f"offsetof.{name}.{f}"]) == getattr(struct, f).offset, (name, f)
+    wl = synth.small_workload("probe", H=3, D=64, T=5, fh=6, fw=7, L=3, wf=1, ws=10, tau=2, mode=0, omega=4)
+    s, p = api.shape_of(wl), api.params_of(wl)
+    assert (int(seen["dims.status"]), int(seen["dims.nQ"]), int(seen["dims.nKmax"])) == (0, *api.rf_schedule_dims(s, p))
+    assert int(seen["workspace_bytes"]) == api.rf_workspace_bytes(s, p)
+    assert int(seen["staging_bytes.3"]) == lib.rf_host_pipeline_staging_bytes(C.byref(s), C.byref(p), 3) > 0
+    assert int(seen["staging_bytes.2"]) == 0
+    assert (int(seen["dims16x32.nQ"]), int(seen["dims16x32.nKmax"])) == api.rf_schedule_dims(s, api.params_of(wl, 16, 32))
+    assert int(seen["bad2d.status"]) == 1 and int(seen["good2d.status"]) == 0 and int(seen["null.status"]) == 1
+    assert int(seen["bounds_checked"]) == lib.rf_bounds_checked()
+    for c in range(8):
+        assert seen[f"status_string.{c}"] == lib.rf_status_string(c).decode()

@@ -246,6 +246,12 @@ rf_status rf_sparse_attn_fwd_plus(const rf_shape *shape, const rf_params *params
  *                                   must be complete in host memory when the call is made.  Returns when the work is
  *                                   enqueued; `wait_stream` (a cudaStream_t, NULL = default stream) is made to wait for
  *                                   the last output copy.  o_host may be read once that stream has been synchronised.
+ *   rf_host_pipeline_set_bandwidths host: candidate bandwidths of the dynamic-bandwidth variant (as for
+ *                                   rf_arm_classify_plus; copied); from the next run on every head takes its own
+ *                                   window.  n_bandwidths = 0 returns to the fixed windows of `params`.
+ *                                   RF_ERR_UNSUPPORTED with params->temporal_window_2d.
+ *   rf_host_pipeline_head_class / _head_window   device int32 [B*H], what ARM decided in the last run (the windows
+ *                                   are written only while bandwidths are set); valid once that run has finished
  *   rf_host_pipeline_status         device int32 the pipeline's kernels report to (dev_status of the calls above)
  *   rf_host_pipeline_destroy        waits for the pipeline's streams, then releases streams and events
  * Errors: RF_ERR_INVALID_ARG (null pointers, head_groups not dividing B*H, misaligned staging), RF_ERR_UNSUPPORTED
@@ -257,6 +263,9 @@ rf_status rf_host_pipeline_create(const rf_shape *shape, const rf_params *params
                                   size_t staging_bytes, rf_host_pipeline **out);
 rf_status rf_host_pipeline_run(rf_host_pipeline *p, const void *q_host, const void *k_host, const void *v_host,
                                void *o_host, void *wait_stream);
+rf_status rf_host_pipeline_set_bandwidths(rf_host_pipeline *p, const float *bandwidths, int32_t n_bandwidths);
+const int32_t *rf_host_pipeline_head_class(rf_host_pipeline *p);
+const int32_t *rf_host_pipeline_head_window(rf_host_pipeline *p);
 int32_t *rf_host_pipeline_status(rf_host_pipeline *p);
 void rf_host_pipeline_destroy(rf_host_pipeline *p);
 

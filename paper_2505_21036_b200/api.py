@@ -23,7 +23,8 @@ EXPORTS = ["rf_status_string", "rf_schedule_dims", "rf_workspace_bytes", "rf_arm
            "rf_build_block_mask", "rf_reorder_tokens", "rf_sparse_attn_fwd", "rf_dense_attn_fwd",
            "rf_arm_classify_noalloc", "rf_selftest_wait_timeout", "rf_arm_classify_plus", "rf_build_block_mask_plus", "rf_sparse_attn_fwd_plus",
            "rf_sparse_attn_reordered", "rf_selftest_arm_abandoned", "rf_bounds_checked", "rf_host_pipeline_staging_bytes",
-           "rf_host_pipeline_create", "rf_host_pipeline_run", "rf_host_pipeline_status", "rf_host_pipeline_destroy"]
+           "rf_host_pipeline_create", "rf_host_pipeline_run", "rf_host_pipeline_status", "rf_host_pipeline_destroy",
+           "rf_host_pipeline_set_bandwidths", "rf_host_pipeline_head_class", "rf_host_pipeline_head_window"]
 
 
 class rf_shape(C.Structure):
@@ -68,6 +69,12 @@ def load():
     lib.rf_host_pipeline_run.argtypes = [V, V, V, V, V, V]
     lib.rf_host_pipeline_status.restype = V
     lib.rf_host_pipeline_status.argtypes = [V]
+    lib.rf_host_pipeline_set_bandwidths.restype = I
+    lib.rf_host_pipeline_set_bandwidths.argtypes = [V, P(C.c_float), C.c_int32]
+    lib.rf_host_pipeline_head_class.restype = V
+    lib.rf_host_pipeline_head_class.argtypes = [V]
+    lib.rf_host_pipeline_head_window.restype = V
+    lib.rf_host_pipeline_head_window.argtypes = [V]
     lib.rf_host_pipeline_destroy.restype = None
     lib.rf_host_pipeline_destroy.argtypes = [V]
     lib.rf_bounds_checked.restype = C.c_int32
@@ -260,6 +267,27 @@ class HostPipeline:
                                            C.byref(h)), "rf_host_pipeline_create")
         self._h = h
         self._status_ptr = lib.rf_host_pipeline_status(h)
+        self._heads = shape.B * shape.H
+
+    def set_bandwidths(self, bandwidths):
+        """Candidate bandwidths of the dynamic-bandwidth variant (empty: back to the fixed windows)."""
+        bw = list(bandwidths)
+        arr = (C.c_float * max(len(bw), 1))(*bw)
+        _check(load().rf_host_pipeline_set_bandwidths(self._h, arr, len(bw)), "rf_host_pipeline_set_bandwidths")
+
+    def _ints(self, ptr):
+        import torch
+        torch.cuda.synchronize()
+        off = ptr - self.staging.data_ptr()
+        return self.staging[off:off + 4 * self._heads].view(torch.int32).cpu().numpy()
+
+    def head_class(self):
+        """ARM's classes of the last run, [B*H] (synchronises)."""
+        return self._ints(load().rf_host_pipeline_head_class(self._h))
+
+    def head_window(self):
+        """The per-head windows of the last run with bandwidths set, [B*H] (synchronises)."""
+        return self._ints(load().rf_host_pipeline_head_window(self._h))
 
     def run(self, qh, kh, vh, oh):
         _check(load().rf_host_pipeline_run(self._h, qh.data_ptr(), kh.data_ptr(), vh.data_ptr(), oh.data_ptr(), _stream()),

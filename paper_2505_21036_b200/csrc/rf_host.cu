@@ -26,6 +26,9 @@ struct rf_host_pipeline {
   size_t ws_bytes;
   rf_schedule sched[2];         // schedule arrays of one group, per compute stream
   int32_t* head_class;          // [groups, heads_per_group]
+  int32_t* head_window;         // the same, written when candidate bandwidths are set (dynamic bandwidth, Sec. 4.3)
+  int n_bw;                     // number of candidate bandwidths, 0: the fixed windows of params
+  float bw[RF_MAX_BANDWIDTHS];
   int32_t* status;
   cudaStream_t s_in, s_run[2], s_out;
   std::vector<cudaEvent_t> landed, run_done, out_done;
@@ -61,7 +64,7 @@ bool layout_of(const rf_shape* shape, const rf_params* params, int groups, rf_sh
   L->head_class = align_up((size_t)heads * sizeof(int32_t));
   L->status = kAlign;
   const size_t lanes = groups > 1 ? 2 : 1;
-  L->total = 4 * L->tensor + lanes * (L->ws + L->count + L->kv_tile + L->kv_len) + L->head_class + L->status;
+  L->total = 4 * L->tensor + lanes * (L->ws + L->count + L->kv_tile + L->kv_len) + 2 * L->head_class + L->status;
   return true;
 }
 
@@ -126,6 +129,8 @@ rf_status rf_host_pipeline_create(const rf_shape* shape, const rf_params* params
     p->sched[r].nKmax = nK;
   }
   p->head_class = reinterpret_cast<int32_t*>(b); b += L.head_class;
+  p->head_window = reinterpret_cast<int32_t*>(b); b += L.head_class;
+  p->n_bw = 0;
   p->status = reinterpret_cast<int32_t*>(b);
   p->s_in = p->s_run[0] = p->s_run[1] = p->s_out = nullptr;
   p->all_done = nullptr;
@@ -158,6 +163,23 @@ void rf_host_pipeline_destroy(rf_host_pipeline* p) {
 }
 
 int32_t* rf_host_pipeline_status(rf_host_pipeline* p) { return p ? p->status : nullptr; }
+const int32_t* rf_host_pipeline_head_class(rf_host_pipeline* p) { return p ? p->head_class : nullptr; }
+const int32_t* rf_host_pipeline_head_window(rf_host_pipeline* p) { return p ? p->head_window : nullptr; }
+
+rf_status rf_host_pipeline_set_bandwidths(rf_host_pipeline* p, const float* bandwidths, int32_t n_bandwidths) {
+  if (p == nullptr || n_bandwidths < 0 || n_bandwidths > RF_MAX_BANDWIDTHS) return RF_ERR_INVALID_ARG;
+  if (n_bandwidths > 0) {
+    if (bandwidths == nullptr) return RF_ERR_INVALID_ARG;
+    if (p->params.temporal_window_2d) return RF_ERR_UNSUPPORTED;
+    for (int i = 0; i < n_bandwidths; ++i) {
+      const float b = bandwidths[i];
+      if (!(b > 0.f && b <= 1.f) || (i > 0 && b <= bandwidths[i - 1])) return RF_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < n_bandwidths; ++i) p->bw[i] = bandwidths[i];
+  }
+  p->n_bw = n_bandwidths;
+  return RF_OK;
+}
 
 rf_status rf_host_pipeline_run(rf_host_pipeline* p, const void* q_host, const void* k_host, const void* v_host, void* o_host,
                                void* wait_stream) {
@@ -181,11 +203,22 @@ rf_status rf_host_pipeline_run(rf_host_pipeline* p, const void* q_host, const vo
     if (p->ran) RF_TRY(cudaStreamWaitEvent(run, p->out_done[g], 0));
     int32_t* hc = p->head_class + (size_t)g * p->heads_per_group;
     const __nv_bfloat16 *q = p->q + g * gelems, *k = p->k + g * gelems, *v = p->v + g * gelems;
-    rf_status st = rf_arm_classify(&p->gshape, &p->params, q, k, hc, nullptr, p->ws[r], p->ws_bytes, p->status, run);
-    if (st == RF_OK) st = rf_build_block_mask(&p->gshape, &p->params, hc, &p->sched[r], p->status, run);
-    if (st == RF_OK)
-      st = rf_sparse_attn_fwd(&p->gshape, &p->params, q, k, v, hc, &p->sched[r], p->o + g * gelems, nullptr, p->ws[r],
-                              p->ws_bytes, p->status, run);
+    rf_status st;
+    if (p->n_bw > 0) {
+      int32_t* hw = p->head_window + (size_t)g * p->heads_per_group;
+      st = rf_arm_classify_plus(&p->gshape, &p->params, p->bw, p->n_bw, q, k, hc, hw, nullptr, p->ws[r], p->ws_bytes, p->status,
+                                run);
+      if (st == RF_OK) st = rf_build_block_mask_plus(&p->gshape, &p->params, hc, hw, &p->sched[r], p->status, run);
+      if (st == RF_OK)
+        st = rf_sparse_attn_fwd_plus(&p->gshape, &p->params, q, k, v, hc, hw, &p->sched[r], p->o + g * gelems, nullptr, p->ws[r],
+                                     p->ws_bytes, p->status, run);
+    } else {
+      st = rf_arm_classify(&p->gshape, &p->params, q, k, hc, nullptr, p->ws[r], p->ws_bytes, p->status, run);
+      if (st == RF_OK) st = rf_build_block_mask(&p->gshape, &p->params, hc, &p->sched[r], p->status, run);
+      if (st == RF_OK)
+        st = rf_sparse_attn_fwd(&p->gshape, &p->params, q, k, v, hc, &p->sched[r], p->o + g * gelems, nullptr, p->ws[r],
+                                p->ws_bytes, p->status, run);
+    }
     if (st != RF_OK) return st;
     RF_TRY(cudaEventRecord(p->run_done[g], run));
     RF_TRY(cudaStreamWaitEvent(p->s_out, p->run_done[g], 0));

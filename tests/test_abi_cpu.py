@@ -123,6 +123,9 @@ def test_host_pipeline_arguments_are_checked_before_cuda(lib):
     assert h.value is None
     assert lib.rf_host_pipeline_run(None, 256, 256, 256, 256, None) == 1
     assert lib.rf_host_pipeline_status(None) is None
+    bw = (C.c_float * 2)(0.25, 0.5)
+    assert lib.rf_host_pipeline_set_bandwidths(None, bw, 2) == 1
+    assert lib.rf_host_pipeline_head_class(None) is None and lib.rf_host_pipeline_head_window(None) is None
     lib.rf_host_pipeline_destroy(None)                 # a no-op
 
 

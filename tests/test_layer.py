@@ -113,3 +113,44 @@ def test_host_staged_calls_back_to_back_with_different_inputs():
         torch.cuda.synchronize()
         assert torch.equal(out.view(torch.int16), o.cpu().view(torch.int16))
     assert not torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+
+
+@pytest.mark.gpu
+def test_host_staged_call_with_dynamic_bandwidth():
+    """The host pipeline with candidate bandwidths set (Sec. 4.3): classes, per-head windows and output equal the
+    resident dynamic-bandwidth entry points bit for bit; invalid lists are refused; clearing the list returns to the
+    fixed windows."""
+    wl, eager = make_layer("cuda", dense_fraction=0.0)
+    shape, params = api.shape_of(wl), api.params_of(wl)
+    pipe = api.HostPipeline(shape, params, "cuda", 2 if (wl.B * wl.H) % 2 == 0 else 1)
+    bws = [0.125, 0.25, 0.5]
+    for bad in ([0.5, 0.25], [0.0], [1.5], [0.1, 0.2, 0.3, 0.4, 0.5]):
+        with pytest.raises(api.RainFusionError):
+            pipe.set_bandwidths(bad)
+    pipe.set_bandwidths(bws)
+    host = [torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in synth.make_qkv(wl)]
+    oh = torch.full(host[0].shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+    pipe.run(*host, oh)
+    assert pipe.status() == 0
+    q, k, v = (t.cuda() for t in host)
+    ws = api.alloc_workspace(shape, params, "cuda")
+    sched = api.Schedule(shape, params, "cuda")
+    hc = torch.zeros((wl.B, wl.H), dtype=torch.int32, device="cuda")
+    hw = torch.zeros((wl.B, wl.H), dtype=torch.int32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = torch.empty_like(q)
+    api.rf_arm_classify_plus(shape, params, bws, q, k, hc, hw, None, ws, st)
+    api.rf_build_block_mask_plus(shape, params, hc, hw, sched, st)
+    api.rf_sparse_attn_fwd_plus(shape, params, q, k, v, hc, hw, sched, o, None, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert np.array_equal(pipe.head_class(), hc.cpu().numpy().reshape(-1))
+    assert np.array_equal(pipe.head_window(), hw.cpu().numpy().reshape(-1))
+    assert torch.equal(oh.view(torch.int16), o.cpu().view(torch.int16))
+    pipe.set_bandwidths([])
+    pipe.run(*host, oh)
+    assert pipe.status() == 0
+    eager(q, k, v, o, None, step=0, num_steps=1)
+    torch.cuda.synchronize()
+    assert torch.equal(oh.view(torch.int16), o.cpu().view(torch.int16))
+    pipe.close()

@@ -96,8 +96,8 @@ class RainFusionAttention:
 
 class HostStagedAttention:
     """The whole path for callers whose Q, K, V and O live in (pinned) host memory: a thin wrapper over the
-    library's rf_host_pipeline_* calls, which pipeline groups of heads over a copy-in, a compute and a copy-out
-    stream (heads are independent at every stage: Algorithm 1 classifies per head; masks and attention are per
+    library's rf_host_pipeline_* calls, which pipeline groups of heads over a copy-in stream, two alternating compute
+    streams and a copy-out stream (heads are independent at every stage: Algorithm 1 classifies per head; masks and attention are per
     head).  Per call every byte of Q, K, V still crosses to the device and every byte of O comes back; only the
     waiting is overlapped, inside a call and between calls made back to back."""
 

@@ -339,6 +339,17 @@ def run_cuda(args, wl):
                          "nominal_peak": f"{NOMINAL_BF16_TFLOPS:.0f} TFLOP/s, NVIDIA's dense bf16 figure for one B200",
                          "algorithmic_flops_per_launch": tile_flops},
         }
+        # The second pipe the kernel leans on: one exponential per score, 16 ex2 per SM and clock (the MUFU pipe: four
+        # lanes per SM sub-partition).  4 * D flops go with every exponential, so at D = 64 this roof, not the tensor
+        # pipe, is the lower one (1191 TFLOP/s at the maximum clock against 2383 at D = 128, where the two meet).
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        exps = 128.0 * 128.0 * listed
+        exp_peak = 16.0 * sms * ((clocks or {}).get("sm_max_mhz") or 1965.0) * 1e6
+        line["roofline"]["exp2"] = {"per_launch": exps, "achieved_per_s": exps / (attn_kernel_ms * 1e-3),
+                                    "peak_per_s": exp_peak, "frac": exps / (attn_kernel_ms * 1e-3) / exp_peak,
+                                    "peak_kind": "16 ex2 per SM per clock at the maximum SM clock",
+                                    "flops_per_exp": 4 * wl.D,
+                                    "roof_tflops": exp_peak * 4 * wl.D / 1e12}
         # the small kernels against the HBM roofline (algorithmic bytes / measured time)
         nS, nT, nX = (int((cls == c).sum()) for c in (0, 1, 2))
         head_bytes = wl.N * wl.D * 2
